@@ -1,0 +1,156 @@
+"""CPU oracle of the ECQ-SGD gradient codec -- TEST INFRASTRUCTURE ONLY.
+
+Thin numpy/ctypes wrapper around ``ecq_oracle.cpp`` (plain single-threaded C++,
+built with ``g++ -O2 -ffp-contract=off``).  Only the tests, the smoke check and
+the CPU-baseline leg of the benchmark may import this package; the CUDA library
+and its Python binding never do, and this package imports nothing of theirs.
+
+Functions follow the paper's Section 4: ``encode`` is Eq. 7 + Eq. 8 (l-infinity
+scale per bucket) + Eq. 9 + Eq. 6 + the fixed-width code; ``decode_mean`` is
+Eq. 4 / the "compute global gradients" line of Algorithm 1.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ecq_oracle.cpp")
+_LIB = os.path.join(_HERE, "libecq_oracle.so")
+
+STATUS_NONFINITE = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (no optimisation that changes fp32 results)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call([
+            "g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math",
+            "-shared", "-fPIC", "-o", tmp, _SRC,
+        ])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        u32, u64, f32, i32 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float, ctypes.c_int
+        vp = ctypes.c_void_p
+        lib.ecqo_philox4x32_10.argtypes = [vp, vp, vp]
+        lib.ecqo_philox4x32_10.restype = None
+        lib.ecqo_draw_word.argtypes = [u64, u32, u32, u64]
+        lib.ecqo_draw_word.restype = u32
+        lib.ecqo_code_bits.argtypes = [u32]
+        lib.ecqo_code_bits.restype = u32
+        lib.ecqo_num_buckets.argtypes = [u64, u32]
+        lib.ecqo_num_buckets.restype = u64
+        lib.ecqo_codes_words.argtypes = [u64, u32]
+        lib.ecqo_codes_words.restype = u64
+        lib.ecqo_encode.argtypes = [u64, u32, u32, f32, f32, u64, i32, u32, u32, u64,
+                                    vp, vp, vp, vp, vp]
+        lib.ecqo_encode.restype = i32
+        lib.ecqo_encode_given_draws.argtypes = [u64, u32, u32, f32, f32, i32,
+                                                vp, vp, vp, vp, vp, vp]
+        lib.ecqo_encode_given_draws.restype = i32
+        lib.ecqo_decode_mean.argtypes = [u64, u32, u32, u32, vp, vp, vp]
+        lib.ecqo_decode_mean.restype = i32
+        lib.ecqo_unpack_levels.argtypes = [u64, u32, vp, vp]
+        lib.ecqo_unpack_levels.restype = None
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def philox4x32_10(ctr: Sequence[int], key: Sequence[int]) -> np.ndarray:
+    """Philox4x32-10 of one 128-bit counter under one 64-bit key (SC'11)."""
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    _load().ecqo_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def draw_word(seed: int, worker: int, step: int, i: int) -> int:
+    """The 32-bit word element ``i`` of ``worker`` draws at iteration ``step``."""
+    return int(_load().ecqo_draw_word(seed, worker, step, i))
+
+
+def code_bits(s: int) -> int:
+    """r = ceil(log2(2s+1)) (paragraph after Eq. 9)."""
+    return int(_load().ecqo_code_bits(s))
+
+
+def num_buckets(d: int, bucket: int) -> int:
+    return int(_load().ecqo_num_buckets(d, bucket))
+
+
+def codes_words(d: int, s: int) -> int:
+    """32-bit words of one worker's code stream."""
+    return int(_load().ecqo_codes_words(d, s))
+
+
+def encode(g: np.ndarray, h: np.ndarray, *, bucket: int, s: int, alpha: float,
+           beta: float, seed: int, worker: int, step: int, mode: int = 0,
+           first_index: int = 0, draws: Optional[np.ndarray] = None):
+    """Encode one worker's slice; ``h`` is updated IN PLACE (Eq. 6).
+
+    Returns ``(codes uint32[words], scales float32[nb], status)``.  ``draws``
+    (one uint32 per element) replaces the Philox stream when given.
+    """
+    assert g.dtype == np.float32 and h.dtype == np.float32
+    assert g.flags.c_contiguous and h.flags.c_contiguous and g.shape == h.shape
+    n = g.size
+    codes = np.zeros(max(codes_words(n, s), 1), dtype=np.uint32)
+    scales = np.zeros(max(num_buckets(n, bucket), 1), dtype=np.float32)
+    status = np.zeros(1, dtype=np.uint32)
+    lib = _load()
+    if draws is None:
+        rc = lib.ecqo_encode(n, bucket, s, alpha, beta, seed, mode, worker, step,
+                             first_index, _ptr(g), _ptr(h), _ptr(codes), _ptr(scales),
+                             _ptr(status))
+    else:
+        dr = np.ascontiguousarray(draws, dtype=np.uint32)
+        assert dr.size == n
+        rc = lib.ecqo_encode_given_draws(n, bucket, s, alpha, beta, mode, _ptr(dr),
+                                         _ptr(g), _ptr(h), _ptr(codes), _ptr(scales),
+                                         _ptr(status))
+    if rc != 0:
+        raise ValueError("oracle encode: bad arguments")
+    return codes[:codes_words(n, s)], scales[:num_buckets(n, bucket)], int(status[0])
+
+
+def decode_mean(codes: Sequence[np.ndarray], scales: Sequence[np.ndarray], *,
+                n: int, bucket: int, s: int) -> np.ndarray:
+    """Mean of the W dequantised messages (Eq. 4)."""
+    W = len(codes)
+    assert W == len(scales) and W >= 1
+    cs = [np.ascontiguousarray(c, dtype=np.uint32) for c in codes]
+    ss = [np.ascontiguousarray(x, dtype=np.float32) for x in scales]
+    cp = (ctypes.c_void_p * W)(*[_ptr(c) for c in cs])
+    sp = (ctypes.c_void_p * W)(*[_ptr(x) for x in ss])
+    out = np.zeros(n, dtype=np.float32)
+    rc = _load().ecqo_decode_mean(n, bucket, s, W, cp, sp, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle decode_mean: bad arguments")
+    return out
+
+
+def unpack_levels(codes: np.ndarray, *, n: int, s: int) -> np.ndarray:
+    """Signed levels q_i in [-s, s] of one message."""
+    c = np.ascontiguousarray(codes, dtype=np.uint32)
+    q = np.zeros(n, dtype=np.int32)
+    _load().ecqo_unpack_levels(n, s, _ptr(c), _ptr(q))
+    return q
