@@ -1,0 +1,162 @@
+/*
+ * ecq.h -- C ABI of the B200 (sm_100a) ECQ-SGD gradient codec.
+ *
+ * The library implements the per-worker, per-iteration codec of "Error
+ * Compensated Quantized SGD" (Wu, Huang, Huang, Zhang, ICML 2018), Section 4,
+ * on a flat fp32 gradient of d entries cut into contiguous buckets of `bucket`
+ * entries (the last bucket may be shorter); each bucket carries its own scale.
+ *
+ * Conventions for every call
+ *   - Returns an int status (ECQ_OK == 0); never throws, never exits.
+ *   - Unless a parameter says "host", data pointers are DEVICE pointers owned
+ *     by the caller; the library never frees or reallocates them.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL
+ *     is the default stream) and the call returns without synchronising,
+ *     unless stated otherwise.
+ *   - `grad`, `err`, `out`, `codes` must be 16-byte aligned; `scales` 4-byte.
+ *   - A context is immutable after creation (except ecq_set_error_mode) and may
+ *     be used from several host threads on different streams.
+ *   - Inputs must be finite.  A bucket whose compensated values contain NaN or
+ *     Inf is sent as all-zero levels with scale 0, its accumulator entries are
+ *     left unchanged, and ECQ_ERR_NONFINITE is recorded in the context's sticky
+ *     device status word (see ecq_status).
+ *
+ * Wire format of one worker's message (paragraph after Eq. 9: r bits per entry
+ * plus one fp32 scale per scaled vector, here per bucket)
+ *   - scales[b], b < nb = ceil(d / bucket): the bucket's l-infinity norm of the
+ *     compensated gradient (0 for an all-zero or non-finite bucket).
+ *   - codes: a dense little-endian bit stream, entry i occupying stream bits
+ *     [i*r, i*r + r), r = ceil(log2(2s+1)); stream bit k is bit (k mod 32) of
+ *     32-bit word (k div 32).  Entry i holds q_i + s, q_i in [-s, s] the signed
+ *     level.  Because bucket % 32 == 0 every bucket starts on a word boundary;
+ *     the stream is padded with zero bits to ecq_codes_words() words.
+ */
+#ifndef ECQ_H_
+#define ECQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ecq_ctx ecq_ctx;
+
+enum {
+    ECQ_OK = 0,
+    ECQ_ERR_ARG = 1,        /* null / misaligned pointer, size or range violation */
+    ECQ_ERR_CUDA = 2,       /* a CUDA runtime or driver call failed */
+    ECQ_ERR_NONFINITE = 3,  /* NaN or Inf met in a compensated gradient (sticky, device) */
+    ECQ_ERR_TIMEOUT = 4,    /* a bounded in-kernel wait on an async copy ran out (sticky, device) */
+    ECQ_ERR_ALLOC = 5       /* host or device allocation failed in ecq_create */
+};
+
+/*
+ * Create a codec context.
+ *   d       entries of the flat gradient (>= 1)
+ *   bucket  entries per bucket: multiple of 32, >= 32
+ *   levels  s of Eq. 9, the number of non-zero quantisation levels, 1..32767
+ *   alpha   compensation coefficient of Eq. 7 (>= 0)
+ *   beta    time-decay factor of Eq. 5/6 (0 <= beta <= 1)
+ *   seed    64-bit key of the Philox4x32-10 stream that drives Eq. 9
+ * The context owns only constants and one 4-byte device status word on the
+ * device that is current at the time of the call.  ECQ_ERR_ARG on a range
+ * violation, ECQ_ERR_ALLOC / ECQ_ERR_CUDA otherwise.
+ */
+int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels,
+               float alpha, float beta, uint64_t seed);
+
+/* Release the context (NULL is allowed).  Synchronises nothing: do not destroy
+ * a context with work in flight. */
+void ecq_destroy(ecq_ctx* ctx);
+
+/*
+ * Choose what the error-accumulator update books.
+ *   0 (default)  Eq. 6 as printed: h <- beta*h + (g - g~), g the raw gradient.
+ *   1            h <- beta*h + ((g + alpha*h) - g~), the compensated value.
+ */
+int ecq_set_error_mode(ecq_ctx* ctx, int mode);
+
+/* r = ceil(log2(2s+1)): bits per entry (paragraph after Eq. 9). */
+uint32_t ecq_code_bits(const ecq_ctx* ctx);
+/* nb = ceil(d / bucket): floats in one worker's `scales`. */
+uint64_t ecq_num_buckets(const ecq_ctx* ctx);
+/* ceil(d*r / 32): 32-bit words in one worker's `codes`. */
+uint64_t ecq_codes_words(const ecq_ctx* ctx);
+
+/*
+ * Sender side, one worker, one iteration (Algorithm 1, "compute quantized local
+ * gradients with Eq. 7" and "update the accumulated quantization error with
+ * Eq. 6", fused):
+ *   v = grad + alpha*err                            (Eq. 7)
+ *   scale_b = max over the bucket of |v_i|          (Eq. 8, l-infinity norm)
+ *   level m_i in {floor(x), floor(x)+1}, x = s|v_i|/scale_b, going up with
+ *   probability x - floor(x), decided by the Philox word of counter
+ *   (i/4, worker, step) under key `seed`            (Eq. 9)
+ *   q_i = sgn(v_i) m_i,  g~_i = q_i * (scale_b / s) (Eq. 8)
+ *   err_i <- beta*err_i + (grad_i - g~_i)           (Eq. 6; see ecq_set_error_mode)
+ *   codes, scales <- the message                    (wire format above)
+ *
+ *   worker, step  identify the random stream; the same (seed, worker, step)
+ *                 always gives the same draws
+ *   grad   [d]    in, never written
+ *   err    [d]    in/out, the accumulator h of this worker; must be zero before
+ *                 the first iteration (h(0) = 0)
+ *   codes  [ecq_codes_words()]  out
+ *   scales [ecq_num_buckets()]  out
+ * Buffers of different workers must not overlap.  ECQ_ERR_ARG on null or
+ * misaligned pointers; ECQ_ERR_CUDA if the launch fails.
+ */
+int ecq_encode(ecq_ctx* ctx, uint32_t worker, uint32_t step, const float* grad,
+               float* err, uint32_t* codes, float* scales, void* cuda_stream);
+
+/*
+ * Receiver side (Eq. 4 and Algorithm 1, "compute global gradients"):
+ *   out_i = (1/W) * sum_{w<W} q_{w,i} * (scales_w[b(i)] / s)
+ *   W       number of messages, 1..ECQ_MAX_WORKERS
+ *   codes   HOST array of W device pointers to the workers' code streams
+ *   scales  HOST array of W device pointers to the workers' scales
+ *   out [d] the averaged dequantised gradient
+ * The two pointer arrays are read before the call returns.
+ */
+#define ECQ_MAX_WORKERS 64
+int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
+                    const float* const* scales, float* out, void* cuda_stream);
+
+/*
+ * One whole iteration from HOST gradients to a HOST result: for every worker
+ * copy its gradient to the device, ecq_encode it, then ecq_decode_mean all W
+ * messages and copy the mean back.  Copies of worker w+1 overlap the encode of
+ * worker w.  The call returns after `out_host` is complete.
+ *   grads_host  HOST array of W HOST pointers, [d] floats each (pinned memory
+ *               makes the copies asynchronous; pageable memory also works)
+ *   err_dev     [W*d] device floats: the W accumulators, worker-major, kept by
+ *               the caller between iterations (zero before the first one)
+ *   workspace_dev, workspace_bytes
+ *               caller-owned device scratch of at least
+ *               ecq_step_host_workspace_bytes(ctx, W) bytes, 256-byte aligned
+ *   out_host    [d] HOST floats
+ */
+uint64_t ecq_step_host_workspace_bytes(const ecq_ctx* ctx, uint32_t W);
+int ecq_step_host(ecq_ctx* ctx, uint32_t W, uint32_t step,
+                  const float* const* grads_host, float* err_dev,
+                  void* workspace_dev, uint64_t workspace_bytes,
+                  float* out_host, void* cuda_stream);
+
+/*
+ * Synchronise `cuda_stream`, then return and clear the context's sticky device
+ * status: ECQ_OK, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT, or ECQ_ERR_CUDA if the
+ * stream itself reports an error.
+ */
+int ecq_status(ecq_ctx* ctx, void* cuda_stream);
+
+/* Number of kernels this library has launched in this process (all contexts). */
+uint64_t ecq_launch_count(void);
+
+/* Static description of a status code. */
+const char* ecq_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ECQ_H_ */

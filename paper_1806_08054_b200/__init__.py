@@ -1,1 +1,13 @@
-"""B200-native ECQ-SGD gradient codec (encode / decode-mean) -- Python binding."""
+"""B200-native ECQ-SGD gradient codec: fused encode and decode-mean kernels.
+
+``binding`` exposes the C ABI of ``include/ecq.h`` under the same names;
+``workloads`` makes the seeded synthetic gradients; ``build`` compiles the
+library in-tree for sm_100a.
+"""
+from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    ECQ_ERR_ARG, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT, ECQ_OK, EcqError, ecq_code_bits,
+    ecq_codes_words, ecq_create, ecq_decode_mean, ecq_destroy, ecq_encode, ecq_launch_count,
+    ecq_num_buckets, ecq_set_error_mode, ecq_status, ecq_step_host,
+    ecq_step_host_workspace_bytes,
+)

@@ -1,0 +1,170 @@
+"""ctypes binding of ``libecq.so``: argument marshalling only.
+
+Every step of the codec runs in the CUDA kernels behind the C ABI declared in
+``include/ecq.h``; the functions here have the same names and only turn torch
+tensors into pointers.  There is no CPU fallback: if the library is missing or a
+tensor is not on a CUDA device the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Sequence
+
+import torch
+
+from .build import LIB
+
+ECQ_OK, ECQ_ERR_ARG, ECQ_ERR_CUDA, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT, ECQ_ERR_ALLOC = range(6)
+ECQ_MAX_WORKERS = 64
+
+_lib = None
+
+
+class EcqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, strerror(status), status))
+
+
+def lib() -> ctypes.CDLL:
+    """Load the compiled library; raise if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB):
+            raise RuntimeError(
+                "libecq.so is not built: run `python -m paper_1806_08054_b200.build` "
+                "(there is no fallback implementation)")
+        L = ctypes.CDLL(LIB)
+        u32, u64, f32, i32, vp = (ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float,
+                                  ctypes.c_int, ctypes.c_void_p)
+        L.ecq_create.argtypes = [ctypes.POINTER(vp), u64, u32, u32, f32, f32, u64]
+        L.ecq_create.restype = i32
+        L.ecq_destroy.argtypes = [vp]
+        L.ecq_destroy.restype = None
+        L.ecq_set_error_mode.argtypes = [vp, i32]
+        L.ecq_set_error_mode.restype = i32
+        L.ecq_code_bits.argtypes = [vp]
+        L.ecq_code_bits.restype = u32
+        L.ecq_num_buckets.argtypes = [vp]
+        L.ecq_num_buckets.restype = u64
+        L.ecq_codes_words.argtypes = [vp]
+        L.ecq_codes_words.restype = u64
+        L.ecq_encode.argtypes = [vp, u32, u32, vp, vp, vp, vp, vp]
+        L.ecq_encode.restype = i32
+        L.ecq_decode_mean.argtypes = [vp, u32, vp, vp, vp, vp]
+        L.ecq_decode_mean.restype = i32
+        L.ecq_step_host_workspace_bytes.argtypes = [vp, u32]
+        L.ecq_step_host_workspace_bytes.restype = u64
+        L.ecq_step_host.argtypes = [vp, u32, u32, vp, vp, vp, u64, vp, vp]
+        L.ecq_step_host.restype = i32
+        L.ecq_status.argtypes = [vp, vp]
+        L.ecq_status.restype = i32
+        L.ecq_launch_count.argtypes = []
+        L.ecq_launch_count.restype = u64
+        L.ecq_strerror.argtypes = [i32]
+        L.ecq_strerror.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().ecq_strerror(status).decode()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (the codec has no CPU path)" % name)
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError("%s must be contiguous %s" % (name, dtype))
+    return t.data_ptr()
+
+
+def ecq_create(d: int, bucket: int, levels: int, alpha: float, beta: float, seed: int) -> int:
+    """Return an opaque context handle (see ``ecq_create`` in ecq.h)."""
+    h = ctypes.c_void_p()
+    rc = lib().ecq_create(ctypes.byref(h), d, bucket, levels, alpha, beta, seed)
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_create")
+    return h.value
+
+
+def ecq_destroy(ctx: int) -> None:
+    lib().ecq_destroy(ctx)
+
+
+def ecq_set_error_mode(ctx: int, mode: int) -> None:
+    rc = lib().ecq_set_error_mode(ctx, mode)
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_set_error_mode")
+
+
+def ecq_code_bits(ctx: int) -> int:
+    return int(lib().ecq_code_bits(ctx))
+
+
+def ecq_num_buckets(ctx: int) -> int:
+    return int(lib().ecq_num_buckets(ctx))
+
+
+def ecq_codes_words(ctx: int) -> int:
+    return int(lib().ecq_codes_words(ctx))
+
+
+def ecq_encode(ctx: int, worker: int, step: int, grad: torch.Tensor, err: torch.Tensor,
+               codes: torch.Tensor, scales: torch.Tensor, stream=None) -> None:
+    """Enqueue the fused sender-side kernel; ``err`` is updated in place."""
+    rc = lib().ecq_encode(ctx, worker, step, _dev(grad, torch.float32, "grad"),
+                          _dev(err, torch.float32, "err"), _dev(codes, torch.int32, "codes"),
+                          _dev(scales, torch.float32, "scales"), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_encode")
+
+
+def ecq_decode_mean(ctx: int, codes: Sequence[torch.Tensor], scales: Sequence[torch.Tensor],
+                    out: torch.Tensor, stream=None) -> None:
+    """Enqueue the fused receiver-side kernel over ``len(codes)`` messages."""
+    W = len(codes)
+    cp = (ctypes.c_void_p * W)(*[_dev(c, torch.int32, "codes") for c in codes])
+    sp = (ctypes.c_void_p * W)(*[_dev(s, torch.float32, "scales") for s in scales])
+    rc = lib().ecq_decode_mean(ctx, W, cp, sp, _dev(out, torch.float32, "out"), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_decode_mean")
+
+
+def ecq_step_host_workspace_bytes(ctx: int, W: int) -> int:
+    return int(lib().ecq_step_host_workspace_bytes(ctx, W))
+
+
+def ecq_step_host(ctx: int, step: int, grads_host: Sequence[torch.Tensor], err: torch.Tensor,
+                  workspace: torch.Tensor, out_host: torch.Tensor, stream=None) -> None:
+    """One iteration from host gradients to a host mean (blocking)."""
+    W = len(grads_host)
+    for g in grads_host:
+        if g.is_cuda or g.dtype != torch.float32 or not g.is_contiguous():
+            raise ValueError("grads_host must be contiguous float32 host tensors")
+    if out_host.is_cuda or out_host.dtype != torch.float32 or not out_host.is_contiguous():
+        raise ValueError("out_host must be a contiguous float32 host tensor")
+    gp = (ctypes.c_void_p * W)(*[g.data_ptr() for g in grads_host])
+    if not workspace.is_cuda:
+        raise ValueError("workspace must be a CUDA tensor")
+    rc = lib().ecq_step_host(ctx, W, step, gp, _dev(err, torch.float32, "err"),
+                             workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                             out_host.data_ptr(), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_step_host")
+
+
+def ecq_status(ctx: int, stream=None) -> int:
+    """Synchronise the stream and return (and clear) the sticky device status."""
+    return int(lib().ecq_status(ctx, _stream(stream)))
+
+
+def ecq_launch_count() -> int:
+    return int(lib().ecq_launch_count())

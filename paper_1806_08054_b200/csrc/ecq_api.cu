@@ -1,0 +1,359 @@
+// C ABI of the ECQ-SGD codec: argument checks, launch configuration, status word.
+#include <atomic>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "../../include/ecq.h"
+#include "ecq_common.cuh"
+#include "ecq_decode.cuh"
+#include "ecq_encode.cuh"
+
+using namespace ecq;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn tensor_map_encoder() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
+                cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+}  // namespace
+
+struct ecq_ctx {
+    CodecParams P;
+    uint64_t nb, n_words;
+    int device;
+    int sm_count;
+    uint32_t* d_status;
+    uint32_t* h_status;          // pinned
+    bool tiled_ok;               // bucket is a power of two <= 4096
+    // lazily created by ecq_step_host
+    std::mutex host_mu;
+    cudaStream_t copy_stream;
+    cudaEvent_t ev_copied[2], ev_encoded[2], ev_start;
+    bool host_ready;
+};
+
+namespace {
+
+// One row of the tiled view is 32 floats; a box is a whole tile of 128 rows.
+bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {32, rows};
+    const cuuint64_t strides[1] = {128};
+    const cuuint32_t box[2] = {32, (cuuint32_t)kTileRows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
+constexpr int kStages = 3;
+
+template <int R>
+int launch_encode_tiled(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
+                        uint32_t* codes, float* scales, cudaStream_t st, uint32_t n_tiles) {
+    using L = EncodeSmem<R, kStages>;
+    static std::once_flag once[16];
+    static int occ[16];
+    const int dev = c->device & 15;
+    auto kern = encode_tiled_kernel<R, kStages>;
+    std::call_once(once[dev], [&] {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        int o = 0;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kEncodeThreads, L::kTotal);
+        occ[dev] = o > 0 ? o : 1;
+    });
+    CUtensorMap tm_g, tm_h;
+    const uint64_t rows = (uint64_t)n_tiles * kTileRows;
+    if (!make_tile_map(&tm_g, g, rows) || !make_tile_map(&tm_h, h, rows)) return ECQ_ERR_CUDA;
+    uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
+    if (grid > n_tiles) grid = n_tiles;
+    kern<<<grid, kEncodeThreads, L::kTotal, st>>>(tm_g, tm_h, c->P, worker, step, g, h, codes,
+                                                  scales, c->d_status, n_tiles);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+int launch_encode_generic(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
+                          uint32_t* codes, float* scales, cudaStream_t st) {
+    const uint64_t want = c->nb;
+    const uint32_t grid = (uint32_t)(want < (uint64_t)c->sm_count * 16 ? want : (uint64_t)c->sm_count * 16);
+    encode_generic_kernel<256><<<grid, 256, 0, st>>>(c->P, worker, step, g, h, codes, scales,
+                                                      c->d_status, 0, c->nb);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+int encode_impl(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
+                uint32_t* codes, float* scales, cudaStream_t st) {
+    const uint32_t n_tiles = c->tiled_ok ? (uint32_t)(c->P.d / kTileElems) : 0;
+    if (n_tiles > 0) {
+        switch (c->P.r) {
+            case 2: return launch_encode_tiled<2>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 3: return launch_encode_tiled<3>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 4: return launch_encode_tiled<4>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 5: return launch_encode_tiled<5>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 6: return launch_encode_tiled<6>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 7: return launch_encode_tiled<7>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 8: return launch_encode_tiled<8>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 9: return launch_encode_tiled<9>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            default: break;
+        }
+    }
+    return launch_encode_generic(c, worker, step, g, h, codes, scales, st);
+}
+
+template <int R>
+void launch_decode(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, cudaStream_t st,
+                   float w_recip, int w_pow2) {
+    constexpr int G = DecodeGroup<R>::kElems;
+    const uint64_t n_groups = (c->P.d + G - 1) / G;
+    uint64_t blocks = (n_groups + 255) / 256;
+    const uint64_t cap = (uint64_t)c->sm_count * 64;
+    if (blocks > cap) blocks = cap;
+    decode_mean_kernel<R><<<(uint32_t)blocks, 256, 0, st>>>(c->P, W, tab, out, n_groups,
+                                                            c->n_words, w_recip, w_pow2);
+}
+
+int decode_impl(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, cudaStream_t st) {
+    const int w_pow2 = (W & (W - 1)) == 0;
+    const float w_recip = 1.0f / (float)W;
+    switch (c->P.r) {
+        case 2: launch_decode<2>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 3: launch_decode<3>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 4: launch_decode<4>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 5: launch_decode<5>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 6: launch_decode<6>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 7: launch_decode<7>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 8: launch_decode<8>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 9: launch_decode<9>(c, W, tab, out, st, w_recip, w_pow2); break;
+        default: {
+            const uint64_t n_groups = (c->P.d + 31) / 32;
+            uint64_t blocks = (n_groups + 255) / 256;
+            const uint64_t cap = (uint64_t)c->sm_count * 64;
+            if (blocks > cap) blocks = cap;
+            decode_mean_generic_kernel<<<(uint32_t)blocks, 256, 0, st>>>(
+                c->P, W, tab, out, n_groups, c->n_words, w_recip, w_pow2);
+        }
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels, float alpha,
+               float beta, uint64_t seed) {
+    if (!out) return ECQ_ERR_ARG;
+    *out = nullptr;
+    if (d == 0 || bucket < 32 || bucket % 32 != 0 || levels == 0 || levels > 32767)
+        return ECQ_ERR_ARG;
+    if (!(alpha >= 0.f) || !(beta >= 0.f) || !(beta <= 1.f) || !(alpha < INFINITY))
+        return ECQ_ERR_ARG;
+    ecq_ctx* c = new (std::nothrow) ecq_ctx();
+    if (!c) return ECQ_ERR_ALLOC;
+    CodecParams& P = c->P;
+    P.d = d; P.bucket = bucket; P.s = levels; P.mode = 0;
+    P.alpha = alpha; P.beta = beta; P.sf = (float)levels;
+    P.r = 0;
+    while ((1ull << P.r) < 2ull * levels + 1ull) ++P.r;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int i = 0; i < 10; ++i) {
+        P.key0[i] = k0; P.key1[i] = k1;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    c->nb = (d + bucket - 1) / bucket;
+    c->n_words = (d * P.r + 31) / 32;
+    c->tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= (uint32_t)kTileElems;
+    c->host_ready = false;
+    c->d_status = nullptr; c->h_status = nullptr;
+    if (cudaGetDevice(&c->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
+        delete c; return ECQ_ERR_CUDA;
+    }
+    if (cudaMalloc(&c->d_status, sizeof(uint32_t)) != cudaSuccess ||
+        cudaMallocHost(&c->h_status, sizeof(uint32_t)) != cudaSuccess) {
+        if (c->d_status) cudaFree(c->d_status);
+        delete c; return ECQ_ERR_ALLOC;
+    }
+    if (cudaMemset(c->d_status, 0, sizeof(uint32_t)) != cudaSuccess) {
+        cudaFree(c->d_status); cudaFreeHost(c->h_status); delete c; return ECQ_ERR_CUDA;
+    }
+    *out = c;
+    return ECQ_OK;
+}
+
+void ecq_destroy(ecq_ctx* c) {
+    if (!c) return;
+    if (c->host_ready) {
+        cudaStreamDestroy(c->copy_stream);
+        for (int i = 0; i < 2; ++i) { cudaEventDestroy(c->ev_copied[i]); cudaEventDestroy(c->ev_encoded[i]); }
+        cudaEventDestroy(c->ev_start);
+    }
+    if (c->d_status) cudaFree(c->d_status);
+    if (c->h_status) cudaFreeHost(c->h_status);
+    delete c;
+}
+
+int ecq_set_error_mode(ecq_ctx* c, int mode) {
+    if (!c || (mode != 0 && mode != 1)) return ECQ_ERR_ARG;
+    c->P.mode = mode;
+    return ECQ_OK;
+}
+
+uint32_t ecq_code_bits(const ecq_ctx* c) { return c ? c->P.r : 0; }
+uint64_t ecq_num_buckets(const ecq_ctx* c) { return c ? c->nb : 0; }
+uint64_t ecq_codes_words(const ecq_ctx* c) { return c ? c->n_words : 0; }
+
+int ecq_encode(ecq_ctx* c, uint32_t worker, uint32_t step, const float* grad, float* err,
+               uint32_t* codes, float* scales, void* cuda_stream) {
+    if (!c || !grad || !err || !codes || !scales) return ECQ_ERR_ARG;
+    if (!aligned16(grad) || !aligned16(err) || !aligned16(codes) || !aligned4(scales))
+        return ECQ_ERR_ARG;
+    return encode_impl(c, worker, step, grad, err, codes, scales,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ecq_decode_mean(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,
+                    const float* const* scales, float* out, void* cuda_stream) {
+    if (!c || !codes || !scales || !out || W == 0 || W > ECQ_MAX_WORKERS) return ECQ_ERR_ARG;
+    if (!aligned16(out)) return ECQ_ERR_ARG;
+    MessageTable tab;
+    std::memset(&tab, 0, sizeof(tab));
+    for (uint32_t w = 0; w < W; ++w) {
+        if (!codes[w] || !scales[w] || !aligned16(codes[w]) || !aligned4(scales[w]))
+            return ECQ_ERR_ARG;
+        tab.codes[w] = codes[w];
+        tab.scales[w] = scales[w];
+    }
+    return decode_impl(c, W, tab, out, static_cast<cudaStream_t>(cuda_stream));
+}
+
+uint64_t ecq_step_host_workspace_bytes(const ecq_ctx* c, uint32_t W) {
+    if (!c || W == 0 || W > ECQ_MAX_WORKERS) return 0;
+    const uint64_t stage = round_up(c->P.d * 4, 256);
+    const uint64_t codes = round_up(c->n_words * 4, 256);
+    const uint64_t scales = round_up(c->nb * 4, 256);
+    return 2 * stage + W * (codes + scales) + stage;
+}
+
+int ecq_step_host(ecq_ctx* c, uint32_t W, uint32_t step, const float* const* grads_host,
+                  float* err_dev, void* workspace_dev, uint64_t workspace_bytes, float* out_host,
+                  void* cuda_stream) {
+    if (!c || !grads_host || !err_dev || !workspace_dev || !out_host || W == 0 ||
+        W > ECQ_MAX_WORKERS)
+        return ECQ_ERR_ARG;
+    if (workspace_bytes < ecq_step_host_workspace_bytes(c, W) ||
+        (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) || !aligned16(err_dev) ||
+        (c->P.d % 4 != 0 && W > 1))     // worker-major accumulators must stay 16-byte aligned
+        return ECQ_ERR_ARG;
+    for (uint32_t w = 0; w < W; ++w)
+        if (!grads_host[w]) return ECQ_ERR_ARG;
+    std::lock_guard<std::mutex> lock(c->host_mu);
+    if (!c->host_ready) {
+        if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+            return ECQ_ERR_CUDA;
+        for (int i = 0; i < 2; ++i) {
+            cudaEventCreateWithFlags(&c->ev_copied[i], cudaEventDisableTiming);
+            cudaEventCreateWithFlags(&c->ev_encoded[i], cudaEventDisableTiming);
+        }
+        cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming);
+        c->host_ready = true;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t d = c->P.d;
+    const uint64_t stage_b = round_up(d * 4, 256);
+    const uint64_t codes_b = round_up(c->n_words * 4, 256);
+    const uint64_t scales_b = round_up(c->nb * 4, 256);
+    uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
+    float* stage[2] = {reinterpret_cast<float*>(ws), reinterpret_cast<float*>(ws + stage_b)};
+    uint8_t* msg = ws + 2 * stage_b;
+    float* out_dev = reinterpret_cast<float*>(msg + W * (codes_b + scales_b));
+
+    MessageTable tab;
+    std::memset(&tab, 0, sizeof(tab));
+    // the copy stream must not run ahead of work already queued on the caller's stream
+    cudaEventRecord(c->ev_start, st);
+    cudaStreamWaitEvent(c->copy_stream, c->ev_start, 0);
+    int rc = ECQ_OK;
+    for (uint32_t w = 0; w < W && rc == ECQ_OK; ++w) {
+        const int sl = w & 1;
+        if (w >= 2) cudaStreamWaitEvent(c->copy_stream, c->ev_encoded[sl], 0);
+        cudaMemcpyAsync(stage[sl], grads_host[w], d * 4, cudaMemcpyHostToDevice, c->copy_stream);
+        cudaEventRecord(c->ev_copied[sl], c->copy_stream);
+        cudaStreamWaitEvent(st, c->ev_copied[sl], 0);
+        uint32_t* codes = reinterpret_cast<uint32_t*>(msg + w * (codes_b + scales_b));
+        float* scales = reinterpret_cast<float*>(msg + w * (codes_b + scales_b) + codes_b);
+        tab.codes[w] = codes;
+        tab.scales[w] = scales;
+        rc = encode_impl(c, w, step, stage[sl], err_dev + (uint64_t)w * d, codes, scales, st);
+        cudaEventRecord(c->ev_encoded[sl], st);
+    }
+    if (rc == ECQ_OK) rc = decode_impl(c, W, tab, out_dev, st);
+    if (rc == ECQ_OK &&
+        cudaMemcpyAsync(out_host, out_dev, d * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        rc = ECQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) rc = ECQ_ERR_CUDA;
+    cudaStreamSynchronize(c->copy_stream);
+    return rc;
+}
+
+int ecq_status(ecq_ctx* c, void* cuda_stream) {
+    if (!c) return ECQ_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(c->h_status, c->d_status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemsetAsync(c->d_status, 0, 4, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return ECQ_ERR_CUDA;
+    const uint32_t bits = *c->h_status;
+    if (bits & kStatusTimeout) return ECQ_ERR_TIMEOUT;
+    if (bits & kStatusNonFinite) return ECQ_ERR_NONFINITE;
+    return ECQ_OK;
+}
+
+uint64_t ecq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* ecq_strerror(int status) {
+    switch (status) {
+        case ECQ_OK: return "ok";
+        case ECQ_ERR_ARG: return "invalid argument (null or misaligned pointer, size or range)";
+        case ECQ_ERR_CUDA: return "a CUDA call failed";
+        case ECQ_ERR_NONFINITE: return "NaN or Inf in a compensated gradient";
+        case ECQ_ERR_TIMEOUT: return "an in-kernel wait on an asynchronous copy ran out";
+        case ECQ_ERR_ALLOC: return "allocation failed";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,257 @@
+"""GPU parity: the CUDA codec, called through its C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_1806_08054_b200 as ecq
+from paper_1806_08054_b200 import workloads as wl
+
+from parity_util import (GpuCodec, SampledOracle, close, codes_np, full_parity, sample_ranges,
+                         whole_vector_properties)
+
+pytestmark = pytest.mark.gpu
+SEED = wl.CODEC_SEED
+
+
+def randn_fn(d, scale=0.01, base=0):
+    def fn(w, t):
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(base + 1000 * t + w)
+        return scale * torch.randn(d, generator=gen, device="cuda")
+    return fn
+
+
+# ------------------------------------------------------------ small shapes ---
+@pytest.mark.parametrize("s", [1, 2, 4, 8, 16, 64, 128, 300, 32767])
+@pytest.mark.parametrize("bucket", [32, 128, 512, 4096, 96, 8192])
+def test_small_shapes_every_width(s, bucket):
+    # several tiles of the tiled kernel plus a ragged end, and the any-shape path
+    sizes = [1, 8, 31, 32, 33, bucket - 1, bucket, bucket + 1, 4096, 3 * 4096 + 5 * 32 + 7]
+    if s in (4, 128):
+        sizes.append(9 * 4096 + bucket + 40)
+    for d in sorted(set(sizes)):
+        full_parity(d, bucket, s, 1.0, 0.9, SEED, W=2, steps=2, grad_fn=randn_fn(d, base=d))
+
+
+@pytest.mark.parametrize("bucket,s", [(512, 4), (2048, 1), (4096, 8), (128, 128), (1024, 2)])
+def test_many_tiles_more_than_one_wave(bucket, s):
+    # more tiles than resident CTAs so that every ring stage is reused
+    d = 4096 * 1500 + 3 * bucket + 24
+    full_parity(d, bucket, s, 1.0, 0.9, SEED, W=1, steps=2, grad_fn=randn_fn(d, base=7),
+                check_decode=True)
+
+
+def test_alpha_beta_variants_and_mode1():
+    d = 4096 * 3 + 777
+    for alpha, beta in ((0.0, 0.0), (0.2, 0.9), (0.01, 1.0), (1.0, 0.99), (2.5, 0.5)):
+        for mode in (0, 1):
+            full_parity(d, 512, 4, alpha, beta, 99, W=2, steps=4, grad_fn=randn_fn(d, base=3),
+                        mode=mode)
+
+
+def test_worker_step_seed_select_the_stream():
+    d, B, s = 8192, 512, 4
+    g = randn_fn(d)(0, 0)
+    outs = {}
+    for seed, worker, step in ((1, 0, 0), (2, 0, 0), (1, 1, 0), (1, 0, 1), (1 << 40, 0, 0)):
+        gpu = GpuCodec(d, B, s, 1.0, 0.9, seed, 1)
+        ecq.ecq_encode(gpu.ctx, worker, step, g, gpu.err[0][1], gpu.codes[0][1], gpu.scales[0][1])
+        assert gpu.status() == 0
+        h = np.zeros(d, np.float32)
+        c_or, _, _ = oracle.encode(g.cpu().numpy(), h, bucket=B, s=s, alpha=1.0, beta=0.9,
+                                   seed=seed, worker=worker, step=step)
+        assert np.array_equal(codes_np(gpu.codes[0][1]), c_or)
+        outs[(seed, worker, step)] = c_or
+        gpu.close()
+    vals = list(outs.values())
+    for i in range(len(vals)):
+        for j in range(i):
+            assert not np.array_equal(vals[i], vals[j])
+
+
+# ------------------------------------------------------------- edge inputs ---
+@pytest.mark.parametrize("bucket", [128, 1024, 4096, 96])
+def test_degenerate_buckets(bucket):
+    d = 4096 * 2 + 3 * bucket + 11
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    g = torch.randn(d, generator=gen, device="cuda")
+    h0 = 0.1 * torch.randn(d, generator=gen, device="cuda")
+    B = bucket
+    g[0:B] = 0; h0[0:B] = 0                       # all-zero bucket
+    g[B:2 * B] = 1e-39; h0[B:2 * B] = 0           # denormal bucket: s/scale overflows
+    g[2 * B] = -0.0; h0[2 * B] = 0                # negative zero among regular entries
+    g[3 * B] = 3.0; g[3 * B + 1] = -3.0; g[3 * B + 2] = 3.0   # ties for the max
+    h0[3 * B:3 * B + 3] = 0
+    g[4 * B - 1] = 50.0                            # max in the last slot
+    g[4 * B] = -60.0                               # max in the first slot
+    g[5 * B:6 * B] = 1e-30                         # tiny but regular scale
+    g[6 * B: 7 * B] = 1e30                         # huge scale
+    full_parity(d, bucket, 4, 1.0, 0.9, SEED, W=1, steps=2, grad_fn=lambda w, t: g, err0=[h0])
+
+
+@pytest.mark.parametrize("bucket", [512, 4096, 96])
+def test_nonfinite_bucket_is_flagged_and_kept(bucket):
+    d = 4096 * 2 + bucket + 5
+    g = randn_fn(d)(0, 0)
+    g[5] = float("nan")
+    g[4096 + 7] = float("inf")
+    g[d - 1] = float("-inf")
+    full_parity(d, bucket, 8, 1.0, 0.9, SEED, W=1, steps=1, grad_fn=lambda w, t: g,
+                expect_status=ecq.ECQ_ERR_NONFINITE)
+    # the sticky status is cleared by reading it
+    gpu = GpuCodec(d, bucket, 8, 1.0, 0.9, SEED, 1)
+    gpu.encode(0, 0, g)
+    assert gpu.status() == ecq.ECQ_ERR_NONFINITE and gpu.status() == ecq.ECQ_OK
+    gpu.close()
+
+
+def test_decode_worker_counts():
+    d, B, s = 4096 * 2 + 100, 512, 4
+    for W in (1, 2, 3, 5, 8, 17, 64):
+        full_parity(d, B, s, 1.0, 0.9, SEED, W=W, steps=1, grad_fn=randn_fn(d, base=W))
+
+
+def test_argument_errors():
+    with pytest.raises(ecq.EcqError):
+        ecq.ecq_create(0, 512, 4, 1.0, 0.9, 1)
+    for bad in ((100, 48, 4, 1.0, 0.9), (100, 512, 0, 1.0, 0.9), (100, 512, 40000, 1.0, 0.9),
+                (100, 512, 4, -1.0, 0.9), (100, 512, 4, 1.0, 1.5), (100, 512, 4, float("nan"), 0.9)):
+        with pytest.raises(ecq.EcqError):
+            ecq.ecq_create(*bad, 1)
+    gpu = GpuCodec(1024, 512, 4, 1.0, 0.9, 1, 1)
+    g = torch.zeros(1025, device="cuda")
+    with pytest.raises(ecq.EcqError):       # misaligned gradient pointer
+        ecq.ecq_encode(gpu.ctx, 0, 0, g[1:], gpu.err[0][1], gpu.codes[0][1], gpu.scales[0][1])
+    with pytest.raises(ValueError):         # host tensor: there is no CPU path
+        ecq.ecq_encode(gpu.ctx, 0, 0, torch.zeros(1024), gpu.err[0][1], gpu.codes[0][1],
+                       gpu.scales[0][1])
+    L = ecq.binding.lib()
+    assert L.ecq_decode_mean(gpu.ctx, 0, None, None, None, None) == ecq.ECQ_ERR_ARG
+    assert L.ecq_decode_mean(gpu.ctx, 65, None, None, None, None) == ecq.ECQ_ERR_ARG
+    gpu.close()
+
+
+def test_checkpoint_resume_is_bit_identical():
+    # the only state is err (+ the caller's step counter)
+    d, B, s = 4096 * 4 + 9, 512, 4
+    fn = randn_fn(d, base=11)
+    a = GpuCodec(d, B, s, 1.0, 0.9, SEED, 1)
+    for t in range(10):
+        a.encode(0, t, fn(0, t))
+    b = GpuCodec(d, B, s, 1.0, 0.9, SEED, 1)
+    for t in range(5):
+        b.encode(0, t, fn(0, t))
+    saved = b.err[0][1].clone()
+    b.close()
+    c = GpuCodec(d, B, s, 1.0, 0.9, SEED, 1)
+    c.err[0][1].copy_(saved)
+    for t in range(5, 10):
+        c.encode(0, t, fn(0, t))
+    assert torch.equal(a.err[0][1], c.err[0][1]) and torch.equal(a.codes[0][1], c.codes[0][1])
+    a.close(); c.close()
+
+
+def test_step_host_matches_device_calls():
+    d, B, s, W = 4096 * 6 + 512 + 8, 512, 4, 5
+    fn = randn_fn(d, base=21)
+    ref = GpuCodec(d, B, s, 1.0, 0.9, SEED, W)
+    ctx = ecq.ecq_create(d, B, s, 1.0, 0.9, SEED)
+    err = torch.zeros(W * d, device="cuda")
+    ws = torch.empty(ecq.ecq_step_host_workspace_bytes(ctx, W), dtype=torch.uint8, device="cuda")
+    out_host = torch.empty(d).pin_memory()
+    for t in range(3):
+        grads = [fn(w, t) for w in range(W)]
+        for w in range(W):
+            ref.encode(w, t, grads[w])
+        ref.decode()
+        hosts = [g.cpu().pin_memory() for g in grads]
+        ecq.ecq_step_host(ctx, t, hosts, err, ws, out_host)
+        assert torch.equal(out_host, ref.out[1].cpu())
+        for w in range(W):
+            assert torch.equal(err[w * d:(w + 1) * d], ref.err[w][1])
+    ecq.ecq_destroy(ctx)
+    ref.close()
+
+
+# --------------------------------------------------- the five configurations --
+def test_config1_gauss_1m_every_element():
+    w = wl.WORKLOADS["gauss_1m"]
+    full_parity(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, w.W, w.steps,
+                lambda p, t: wl.gradient(w, p, t, "cuda"))
+
+
+def _sampled_config(w, steps, W=None, ranges=None, grads=None):
+    """Full-size run; the oracle follows sampled whole-bucket ranges, and
+    whole-vector properties are checked on the device."""
+    W = W or w.W
+    ranges = ranges or sample_ranges(w.d, w.bucket, seed=w.index)
+    gpu = GpuCodec(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, W)
+    so = SampledOracle(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, W, ranges)
+    try:
+        for t in range(steps):
+            for p in range(W):
+                g = grads(p, t) if grads else wl.gradient(w, p, t, "cuda")
+                before = gpu.err[p][1].clone() if p == 0 else None
+                gpu.encode(p, t, g)
+                if p == 0:
+                    whole_vector_properties(gpu, p, g, before, w.alpha)
+                so.encode_and_compare(gpu, p, t, g)
+                del g
+            gpu.decode(W)
+            assert gpu.status() == ecq.ECQ_OK
+            so.decode_and_compare(gpu)
+            gpu.check_guards()
+    finally:
+        gpu.close()
+        wl.clear_cache()
+        torch.cuda.empty_cache()
+
+
+def test_config2_lsq_4m():
+    w = wl.WORKLOADS["lsq_4m"]
+    _sampled_config(w, steps=w.steps)
+
+
+def test_config3_resnet50():
+    w = wl.WORKLOADS["resnet50"]
+    _sampled_config(w, steps=w.steps)
+
+
+def test_config4_alexnet():
+    w = wl.WORKLOADS["alexnet"]
+    _sampled_config(w, steps=w.steps)
+
+
+@pytest.mark.parametrize("bucket", wl.LM_SWEEP_BUCKETS)
+@pytest.mark.parametrize("s", wl.LM_SWEEP_LEVELS)
+def test_config5_lm_350m_sweep(bucket, s):
+    base = wl.WORKLOADS["lm_350m"]
+    w = wl.with_codec(base, bucket, s)
+    free, _ = torch.cuda.mem_get_info()
+    need = (w.W * w.d * 4) + 4 * w.d * 4 + w.W * w.d * 9 // 8 + 6 * w.d * 4
+    if free < need * 1.05:
+        pytest.skip("needs %.0f GB of free device memory" % (need / 1e9))
+    # four distinct gradient buffers per step; worker p reads buffer p mod 4
+    # (its Philox stream and its accumulator are still its own)
+    cache = {}
+
+    def grads(p, t):
+        key = (p % 4, t)
+        if key not in cache:
+            for k in [k for k in cache if k[1] != t]:
+                del cache[k]
+            cache[key] = wl.gradient(w, p % 4, t, "cuda")
+        return cache[key]
+    steps = w.steps if (bucket, s) == (512, 4) else 1
+    _sampled_config(w, steps=steps, grads=grads)
+    cache.clear()
+    torch.cuda.empty_cache()
+
+
+def test_code_width_matched_levels_on_resnet50():
+    # the quantiser whose 2s+1 levels exactly fill b bits: s = 2^(b-1) - 1
+    base = wl.WORKLOADS["resnet50"]
+    for s in (3, 7, 127):
+        _sampled_config(wl.with_codec(base, base.bucket, s), steps=1, W=2)
