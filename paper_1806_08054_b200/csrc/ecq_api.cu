@@ -74,22 +74,23 @@ bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
            CUDA_SUCCESS;
 }
 
-constexpr int kStages = 3;
-
 template <int R>
 int launch_encode_tiled(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
                         uint32_t* codes, float* scales, cudaStream_t st, uint32_t n_tiles) {
-    using L = EncodeSmem<R, kStages>;
+    using L = EncodeSmem<R>;
     static std::once_flag once[16];
     static int occ[16];
     const int dev = c->device & 15;
-    auto kern = encode_tiled_kernel<R, kStages>;
+    auto kern = encode_tiled_kernel<R>;
     std::call_once(once[dev], [&] {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
         int o = 0;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kEncodeThreads, L::kTotal);
-        occ[dev] = o > 0 ? o : 1;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) ==
+                cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kEncodeThreads, L::kTotal) ==
+                cudaSuccess)
+            occ[dev] = o;
     });
+    if (occ[dev] <= 0) return ECQ_ERR_CUDA;
     CUtensorMap tm_g, tm_h;
     const uint64_t rows = (uint64_t)n_tiles * kTileRows;
     if (!make_tile_map(&tm_g, g, rows) || !make_tile_map(&tm_h, h, rows)) return ECQ_ERR_CUDA;
@@ -195,7 +196,7 @@ int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels, floa
     }
     c->nb = (d + bucket - 1) / bucket;
     c->n_words = (d * P.r + 31) / 32;
-    c->tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= (uint32_t)kTileElems;
+    c->tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= kMaxTiledBucket;
     c->host_ready = false;
     c->d_status = nullptr; c->h_status = nullptr;
     if (cudaGetDevice(&c->device) != cudaSuccess ||

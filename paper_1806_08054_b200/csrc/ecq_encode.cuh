@@ -116,220 +116,217 @@ encode_generic_kernel(CodecParams P, uint32_t worker, uint32_t step, const float
 }
 
 // ===========================================================================
-// Tiled path.  The vector is seen as a matrix of 128-byte rows (32 floats).  A
+// Tiled path.  The vector is seen as a matrix of 128-byte rows (32 floats); a
 // tile is 128 rows = 4096 entries = a whole number of buckets (bucket a power
-// of two <= 4096).  A persistent CTA streams its tiles through an NSTAGES ring
-// in shared memory:
-//   producer lane : TMA loads of the g and h tiles (128-byte swizzle) ->
-//                   full[s];  after the consumers are done with a stage it
-//                   issues the TMA store of the updated h tile and a linear
-//                   bulk store of the tile's code words, then refills the stage
-//   128 consumers : one thread per row.  The swizzle makes a thread's eight
-//                   16-byte chunks of its row conflict-free across the warp.
-//                   Pass 1 takes the row max, the rows of a bucket are combined
-//                   by shuffles (and one shared-memory hop above 1024 entries);
-//                   pass 2 re-reads the row, draws Philox per 4 entries, rounds,
-//                   updates h in place and packs the 32 codes into R words.
+// of two <= 4096).  A persistent CTA of 128 threads (four per SM) owns one
+// 32 KiB load buffer and one store staging buffer and walks its tiles:
+//   * thread 0 issues two 16 KiB TMA loads (g and h tile, 128-byte swizzle);
+//     measured on B200, a TMA operation costs ~200 cycles of issue time
+//     whatever its size, so tiles are moved with few large operations;
+//   * every thread copies its row of g and h to registers (the swizzle makes
+//     the eight 16-byte chunks of a row conflict-free across the warp); after
+//     one CTA barrier the buffer is refilled with the next tile, which lands
+//     while this one is being computed;
+//   * the row max of |g + alpha h| is combined over the rows of a bucket by
+//     shuffles (and through shared memory when a bucket spans 2 or 4 warps);
+//   * each thread draws Philox per 4 entries, rounds, forms the new h row in
+//     registers and packs its 32 codes into R words; both go to the staging
+//     buffer, from which thread 0 issues one TMA store (h tile) and one linear
+//     bulk store (code words).
 // g and h are read from HBM once, h is written once; v never leaves the SM.
 // ===========================================================================
 constexpr int kTileRows = 128;
 constexpr int kTileElems = kTileRows * 32;          // 4096
 constexpr int kTileBytes = kTileElems * 4;          // 16 KiB per operand
-constexpr int kConsumers = kTileRows;               // one thread per row
-constexpr int kEncodeThreads = kConsumers + 32;     // + producer warp
+constexpr int kEncodeThreads = kTileRows;           // one thread per row
+constexpr int kEncodeCtasPerSm = 4;
+constexpr uint32_t kMaxTiledBucket = kTileElems;    // largest bucket of the tiled path
 
-template <int R, int NSTAGES>
+template <int R>
 struct EncodeSmem {
-    static constexpr int kCodeBytes = R * (kTileElems / 8);       // R * 512
-    static constexpr int kStageBytes = 2 * kTileBytes;
-    static constexpr int kCodesOff = NSTAGES * kStageBytes;
-    static constexpr int kBarOff = kCodesOff + NSTAGES * kCodeBytes;
-    static constexpr int kMiscOff = kBarOff + 2 * NSTAGES * 8;
-    static constexpr int kTotal = kMiscOff + 64 + 1024;           // + alignment slack
+    static constexpr int kCodeBytes = R * (kTileElems / 8);       // R * 512 per tile
+    static constexpr int kLoadOff = 0;                            // g tile, h tile
+    static constexpr int kHoutOff = 2 * kTileBytes;               // staged new h tile
+    static constexpr int kCoutOff = 3 * kTileBytes;               // staged code words
+    static constexpr int kBarOff = kCoutOff + kCodeBytes;
+    static constexpr int kMiscOff = kBarOff + 16;
+    static constexpr int kTotal = kMiscOff + 48 + 1024;           // + alignment slack
 };
 
-template <int R, int NSTAGES>
-__global__ void __launch_bounds__(kEncodeThreads)
+// max(m, |a|, |b|) that returns NaN if any input is NaN
+__device__ __forceinline__ float max3_abs_nan(float m, float a, float b) {
+    float r;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b)));
+    return r;
+}
+
+template <int R>
+__global__ void __launch_bounds__(kEncodeThreads, kEncodeCtasPerSm)
 encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_h,
                     const CodecParams P, const uint32_t worker, const uint32_t step,
                     const float* __restrict__ g, float* h, uint32_t* __restrict__ codes,
                     float* __restrict__ scales, uint32_t* status, const uint32_t n_tiles) {
-    using L = EncodeSmem<R, NSTAGES>;
+    using L = EncodeSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* const sm = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bar_full = base + L::kBarOff;
-    const uint32_t bar_done = bar_full + NSTAGES * 8;
     volatile uint32_t* s_abort = reinterpret_cast<volatile uint32_t*>(sm + L::kMiscOff);
-    uint32_t* s_wmax = reinterpret_cast<uint32_t*>(sm + L::kMiscOff + 16);   // 4 warps x 2 parities
+    uint32_t* s_wmax = reinterpret_cast<uint32_t*>(sm + L::kMiscOff + 16);   // one per warp
 
     const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    auto issue_load = [&](uint32_t tile) {
+        mbar_arrive_expect_tx(bar_full, 2 * kTileBytes);
+        tma_load_2d(base + L::kLoadOff, &tm_g, 0, (int)(tile * kTileRows), bar_full);
+        tma_load_2d(base + L::kLoadOff + kTileBytes, &tm_h, 0, (int)(tile * kTileRows), bar_full);
+    };
     if (tid == 0) {
-        for (int s = 0; s < NSTAGES; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_done + 8 * s, kConsumers);
-        }
+        mbar_init(bar_full, 1);
         *s_abort = 0;
         fence_mbar_init();
+        if (blockIdx.x < n_tiles) issue_load(blockIdx.x);
     }
     __syncthreads();
 
-    const uint32_t n_my = (n_tiles > blockIdx.x)
-                              ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    const uint32_t rpb = P.bucket >> 5;              // rows per bucket, power of two <= 128
+    const uint32_t sw = (uint32_t)(tid & 7) << 4;
+    const uint32_t rpb = P.bucket >> 5;                    // rows per bucket, power of two <= 128
+    const uint32_t buckets_per_tile = kTileElems / P.bucket;
+    const float magic_code = 12582912.f + P.sf;            // 1.5*2^23 + s, exact
+    const uint8_t* const g_row = sm + L::kLoadOff + tid * 128;
+    const uint8_t* const h_row = g_row + kTileBytes;
+    uint8_t* const hout_row = sm + L::kHoutOff + tid * 128;
+    uint32_t* const cout_row = reinterpret_cast<uint32_t*>(sm + L::kCoutOff) + tid * R;
 
-    if (tid >= kConsumers) {
-        // ------------------------------ producer ------------------------------
-        if (tid == kConsumers) {
-            auto issue_load = [&](uint32_t k) {
-                const uint32_t s = k % NSTAGES;
-                const uint32_t tile = blockIdx.x + k * gridDim.x;
-                const uint32_t bar = bar_full + 8 * s;
-                mbar_arrive_expect_tx(bar, 2 * kTileBytes);
-                tma_load_2d(base + s * L::kStageBytes, &tm_g, 0, (int)(tile * kTileRows), bar);
-                tma_load_2d(base + s * L::kStageBytes + kTileBytes, &tm_h, 0,
-                            (int)(tile * kTileRows), bar);
-            };
-            uint32_t issued = 0;
-            for (; issued < n_my && issued < (uint32_t)NSTAGES; ++issued) issue_load(issued);
-            bool ok = true;
-            for (uint32_t k = 0; k < n_my; ++k) {
-                const uint32_t s = k % NSTAGES;
-                if (*s_abort || !mbar_wait(bar_done + 8 * s, (k / NSTAGES) & 1u)) { ok = false; break; }
-                const uint32_t tile = blockIdx.x + k * gridDim.x;
-                tma_store_2d(&tm_h, 0, (int)(tile * kTileRows),
-                             base + s * L::kStageBytes + kTileBytes);
-                bulk_store_1d(codes + (uint64_t)tile * (R * kTileRows),
-                              base + L::kCodesOff + s * L::kCodeBytes, L::kCodeBytes);
-                bulk_commit();
-                if (issued < n_my) {
-                    bulk_wait_read0();               // the stage is free once the stores have read it
-                    issue_load(issued++);
-                }
-            }
-            if (!ok) {
-                *s_abort = 1;
-                atomicOr(status, kStatusTimeout);
-                // let the loads still in flight land before the CTA gives up its shared memory
-                const uint32_t first = issued > (uint32_t)NSTAGES ? issued - NSTAGES : 0;
-                for (uint32_t j = first; j < issued; ++j)
-                    mbar_wait(bar_full + 8 * (j % NSTAGES), (j / NSTAGES) & 1u);
-            }
-            bulk_wait_all();
+    uint32_t parity = 0;
+    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, parity ^= 1u) {
+        if (!mbar_wait(bar_full, parity)) { *s_abort = 1; atomicOr(status, kStatusTimeout); }
+
+        // my row of g and h -> registers
+        float4 G[8], H[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t off = ((uint32_t)c << 4) ^ sw;
+            G[c] = *reinterpret_cast<const float4*>(g_row + off);
+            H[c] = *reinterpret_cast<const float4*>(h_row + off);
         }
-    } else {
-        // ------------------------------ consumers -----------------------------
-        const int row = tid;
-        const int lane = tid & 31;
-        const int warp = tid >> 5;
-        const uint32_t sw = (uint32_t)(row & 7) << 4;
-        const uint32_t buckets_per_tile = kTileElems / P.bucket;
-        for (uint32_t k = 0; k < n_my; ++k) {
-            const uint32_t s = k % NSTAGES;
-            const uint32_t tile = blockIdx.x + k * gridDim.x;
-            bool ok = mbar_wait(bar_full + 8 * s, (k / NSTAGES) & 1u);
-            if (!ok) { *s_abort = 1; atomicOr(status, kStatusTimeout); }
-            const uint8_t* gs = sm + s * L::kStageBytes + row * 128;
-            uint8_t* hs = sm + s * L::kStageBytes + kTileBytes + row * 128;
+        // row max of |g + alpha h| (NaN-propagating), then over the rows of the bucket
+        float mf = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            mf = max3_abs_nan(mf, __fmaf_rn(P.alpha, H[c].x, G[c].x), __fmaf_rn(P.alpha, H[c].y, G[c].y));
+            mf = max3_abs_nan(mf, __fmaf_rn(P.alpha, H[c].z, G[c].z), __fmaf_rn(P.alpha, H[c].w, G[c].w));
+        }
+        // non-negative floats and NaN (0x7FFFFFFF) order like their bit patterns
+        uint32_t m = __float_as_uint(mf) & 0x7FFFFFFFu;
+        for (uint32_t o = 1; o < rpb && o < 32; o <<= 1)
+            m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        if (rpb > 32 && lane == 0) s_wmax[warp] = m;
+        // the stores of the previous tile must have read the staging buffer
+        if (tid == 0) bulk_wait_read0();
+        __syncthreads();                                   // load buffer and staging are free
+        if (*s_abort) break;                               // uniform: set before the barrier
+        if (tid == 0 && tile + gridDim.x < n_tiles) issue_load(tile + gridDim.x);
+        if (rpb == 64) m = max(s_wmax[warp & ~1], s_wmax[warp | 1]);
+        if (rpb == 128) m = max(max(s_wmax[0], s_wmax[1]), max(s_wmax[2], s_wmax[3]));
+        const BucketScale bs = bucket_scale(m, P.sf);
+        if ((tid & (rpb - 1)) == 0) {
+            scales[(uint64_t)tile * buckets_per_tile + tid / rpb] = bs.scale;
+            if (bs.kind == 2) atomicOr(status, kStatusNonFinite);
+        }
 
-            // pass 1: row max of |g + alpha h|
-            uint32_t m = 0;
+        // round, new h (kept in H), pack 32 codes into R words.  The codes enter a
+        // 64-bit window as (float bits of q + s + 1.5*2^23) << pos; the constant
+        // high bits are removed once per output word.
+        const uint64_t blk0 = (uint64_t)tile * (kTileElems / 4) + (uint32_t)tid * 8;
+        uint32_t wout[R];
+        uint64_t acc = 0, junk = 0;
+        int nbits = 0, kw = 0;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t off = ((uint32_t)c << 4) ^ sw;
-                const float4 g4 = *reinterpret_cast<const float4*>(gs + off);
-                const float4 h4 = *reinterpret_cast<const float4*>(hs + off);
-                m = max(m, __float_as_uint(__fmaf_rn(P.alpha, h4.x, g4.x)) & 0x7FFFFFFFu);
-                m = max(m, __float_as_uint(__fmaf_rn(P.alpha, h4.y, g4.y)) & 0x7FFFFFFFu);
-                m = max(m, __float_as_uint(__fmaf_rn(P.alpha, h4.z, g4.z)) & 0x7FFFFFFFu);
-                m = max(m, __float_as_uint(__fmaf_rn(P.alpha, h4.w, g4.w)) & 0x7FFFFFFFu);
-            }
-            // combine the rows of a bucket
-            for (uint32_t o = 1; o < rpb && o < 32; o <<= 1)
-                m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-            if (rpb > 32) {
-                uint32_t* wm = s_wmax + (k & 1u) * 4;
-                if (lane == 0) wm[warp] = m;
-                named_bar_sync(1, kConsumers);
-                if (rpb == 64) m = max(wm[warp & ~1], wm[warp | 1]);
-                else m = max(max(wm[0], wm[1]), max(wm[2], wm[3]));
-                if (*s_abort) break;                 // uniform: read after the barrier
-            } else {
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;                      // warp-uniform
-            }
-            const BucketScale bs = bucket_scale(m, P.sf);
-            if ((row & (rpb - 1)) == 0) {
-                scales[(uint64_t)tile * buckets_per_tile + row / rpb] = bs.scale;
-                if (bs.kind == 2) atomicOr(status, kStatusNonFinite);
-            }
-
-            // pass 2: round, update h in place, pack 32 codes into R words
-            const uint64_t blk0 = (uint64_t)tile * (kTileElems / 4) + (uint32_t)row * 8;
-            uint32_t wout[R];
-            uint64_t acc = 0;
-            int nbits = 0, kw = 0;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t off = ((uint32_t)c << 4) ^ sw;
-                const float4 g4 = *reinterpret_cast<const float4*>(gs + off);
-                const float4 h4 = *reinterpret_cast<const float4*>(hs + off);
-                const float gv[4] = {g4.x, g4.y, g4.z, g4.w};
-                const float hv[4] = {h4.x, h4.y, h4.z, h4.w};
-                float hn[4];
-                uint32_t code[4];
-                if (bs.kind == 0) {
-                    uint32_t Rw[4];
-                    const uint64_t blk = blk0 + c;
-                    philox4x32_10(P, (uint32_t)blk, (uint32_t)(blk >> 32), worker, step, Rw);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float v = __fmaf_rn(P.alpha, hv[j], gv[j]);
-                        code[j] = quantise_entry(gv[j], hv[j], v, Rw[j], bs, P, hn[j]);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float v = __fmaf_rn(P.alpha, hv[j], gv[j]);
-                        code[j] = P.s;
-                        hn[j] = (bs.kind == 1) ? __fmaf_rn(P.beta, hv[j], P.mode ? v : gv[j]) : hv[j];
-                    }
-                }
-                *reinterpret_cast<float4*>(hs + off) = make_float4(hn[0], hn[1], hn[2], hn[3]);
+        for (int c = 0; c < 8; ++c) {
+            const float gv[4] = {G[c].x, G[c].y, G[c].z, G[c].w};
+            const float hv[4] = {H[c].x, H[c].y, H[c].z, H[c].w};
+            float hn[4];
+            uint32_t cb[4];
+            if (bs.kind == 0) {
+                uint32_t Rw[4];
+                const uint64_t blk = blk0 + c;
+                philox4x32_10(P, (uint32_t)blk, (uint32_t)(blk >> 32), worker, step, Rw);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    acc |= (uint64_t)code[j] << nbits;
-                    nbits += R;
-                    if (nbits >= 32) { wout[kw++] = (uint32_t)acc; acc >>= 32; nbits -= 32; }
+                    const float v = __fmaf_rn(P.alpha, hv[j], gv[j]);
+                    const uint32_t sgn = __float_as_uint(v) & 0x80000000u;
+                    const float x = fminf(__fmul_rn(fabsf(v), bs.inv), P.sf);
+                    const float lf = __fsub_rn(__fadd_rz(x, 8388608.f), 8388608.f);   // floor
+                    const float f = __fsub_rn(x, lf);
+                    const float u = __fmul_rn(__uint2float_rn(Rw[j] >> 8), 0x1p-24f);
+                    const float mlev = __fadd_rn(lf, (u < f) ? 1.f : 0.f);
+                    // work on sgn(v)*g so that the level stays non-negative: negation
+                    // commutes with rounding, and a zero level leaves g untouched
+                    const float gsn = __uint_as_float(__float_as_uint(P.mode ? v : gv[j]) ^ sgn);
+                    const float esn = __fsub_rn(gsn, __fmul_rn(mlev, bs.a));
+                    const float e = __uint_as_float(__float_as_uint(esn) ^ sgn);
+                    hn[j] = __fmaf_rn(P.beta, hv[j], e);
+                    const float q = __uint_as_float(__float_as_uint(mlev) ^ sgn);
+                    cb[j] = __float_as_uint(__fadd_rn(q, magic_code));     // 0x4B400000 + q + s
                 }
-            }
-            uint32_t* cs = reinterpret_cast<uint32_t*>(sm + L::kCodesOff + s * L::kCodeBytes) + row * R;
-            if constexpr (R % 4 == 0) {
-#pragma unroll
-                for (int q = 0; q < R / 4; ++q)
-                    reinterpret_cast<uint4*>(cs)[q] =
-                        make_uint4(wout[4 * q], wout[4 * q + 1], wout[4 * q + 2], wout[4 * q + 3]);
-            } else if constexpr (R % 2 == 0) {
-#pragma unroll
-                for (int q = 0; q < R / 2; ++q)
-                    reinterpret_cast<uint2*>(cs)[q] = make_uint2(wout[2 * q], wout[2 * q + 1]);
             } else {
 #pragma unroll
-                for (int q = 0; q < R; ++q) cs[q] = wout[q];
+                for (int j = 0; j < 4; ++j) {
+                    const float v = __fmaf_rn(P.alpha, hv[j], gv[j]);
+                    cb[j] = 0x4B400000u + P.s;
+                    hn[j] = (bs.kind == 1) ? __fmaf_rn(P.beta, hv[j], P.mode ? v : gv[j]) : hv[j];
+                }
             }
-            fence_proxy_async_smem();               // my writes -> visible to the TMA stores
-            mbar_arrive(bar_done + 8 * s);
+            *reinterpret_cast<float4*>(hout_row + (((uint32_t)c << 4) ^ sw)) =
+                make_float4(hn[0], hn[1], hn[2], hn[3]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc += (uint64_t)cb[j] * (uint64_t)(1u << nbits);
+                junk += (uint64_t)0x4B400000u << nbits;
+                nbits += R;
+                if (nbits >= 32) {
+                    acc -= junk; junk = 0;
+                    wout[kw++] = (uint32_t)acc;
+                    acc >>= 32;
+                    nbits -= 32;
+                }
+            }
+        }
+        if constexpr (R % 4 == 0) {
+#pragma unroll
+            for (int q = 0; q < R / 4; ++q)
+                reinterpret_cast<uint4*>(cout_row)[q] =
+                    make_uint4(wout[4 * q], wout[4 * q + 1], wout[4 * q + 2], wout[4 * q + 3]);
+        } else if constexpr (R % 2 == 0) {
+#pragma unroll
+            for (int q = 0; q < R / 2; ++q)
+                reinterpret_cast<uint2*>(cout_row)[q] = make_uint2(wout[2 * q], wout[2 * q + 1]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < R; ++q) cout_row[q] = wout[q];
+        }
+        fence_proxy_async_smem();               // my writes -> visible to the TMA stores
+        __syncthreads();
+        if (tid == 0) {
+            tma_store_2d(&tm_h, 0, (int)(tile * kTileRows), base + L::kHoutOff);
+            bulk_store_1d(codes + (uint64_t)tile * (R * kTileRows), base + L::kCoutOff, L::kCodeBytes);
+            bulk_commit();
         }
     }
-
+    if (tid == 0) {
+        if (*s_abort) mbar_wait(bar_full, parity);   // let a load still in flight land
+        bulk_wait_all();
+    }
     __syncthreads();
     if (*s_abort) return;
 
-    // ragged end: the buckets after the last whole tile, spread over the CTAs
-    // from the back of the grid (those own one tile fewer)
-    const uint64_t tail_first = (uint64_t)n_tiles * (kTileElems / P.bucket);
+    // ragged end: the buckets after the last whole tile, spread over the CTAs from
+    // the back of the grid
+    const uint64_t tail_first = (uint64_t)n_tiles * buckets_per_tile;
     const uint64_t nb_total = (P.d + P.bucket - 1) / P.bucket;
-    uint32_t* s_red = reinterpret_cast<uint32_t*>(sm);   // the ring is idle now
+    uint32_t* s_red = reinterpret_cast<uint32_t*>(sm);   // the buffers are idle now
     for (uint64_t b = tail_first + (gridDim.x - 1 - blockIdx.x); b < nb_total; b += gridDim.x)
         encode_bucket_generic<kEncodeThreads>(P, b, worker, step, g, h, codes, scales, status,
                                               s_red, tid);
