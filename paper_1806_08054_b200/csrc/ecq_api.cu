@@ -143,10 +143,54 @@ void launch_decode(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, 
                                                             c->n_words, w_recip, w_pow2);
 }
 
+// Tiled decode: returns false when the shape is not covered (caller falls back).
+template <int R>
+bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out,
+                         cudaStream_t st, float w_recip, int w_pow2) {
+    using L = DecodeTiled<R>;
+    const uint32_t B = c->P.bucket;
+    const uint64_t n_tiles64 = c->P.d / kDecTileElems;
+    if ((B & (B - 1)) != 0 || n_tiles64 == 0 || n_tiles64 > 0xFFFFFFFFull) return false;
+    const uint32_t gsz = B >= 1024 ? 32 : B / 32;
+    if (W > (uint32_t)kDecAreg * gsz) return false;
+    static std::once_flag once[16];
+    static int occ[16];
+    const int dev = c->device & 15;
+    auto kern = decode_tiled_kernel<R>;
+    std::call_once(once[dev], [&] {
+        int o = 0;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmem) ==
+                cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kDecWarps * 32, L::kSmem) ==
+                cudaSuccess)
+            occ[dev] = o;
+    });
+    if (occ[dev] <= 0) return false;
+    const uint32_t n_tiles = (uint32_t)n_tiles64;
+    uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
+    const uint32_t want = (n_tiles + kDecWarps - 1) / kDecWarps;
+    if (grid > want) grid = want;
+    kern<<<grid, kDecWarps * 32, L::kSmem, st>>>(c->P, W, tab, out, n_tiles, c->n_words, w_recip,
+                                                 w_pow2);
+    return true;
+}
+
 int decode_impl(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, cudaStream_t st) {
     const int w_pow2 = (W & (W - 1)) == 0;
     const float w_recip = 1.0f / (float)W;
+    bool done = false;
     switch (c->P.r) {
+        case 2: done = launch_decode_tiled<2>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 3: done = launch_decode_tiled<3>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 4: done = launch_decode_tiled<4>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 5: done = launch_decode_tiled<5>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 6: done = launch_decode_tiled<6>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 7: done = launch_decode_tiled<7>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 8: done = launch_decode_tiled<8>(c, W, tab, out, st, w_recip, w_pow2); break;
+        case 9: done = launch_decode_tiled<9>(c, W, tab, out, st, w_recip, w_pow2); break;
+        default: break;
+    }
+    if (!done) switch (c->P.r) {
         case 2: launch_decode<2>(c, W, tab, out, st, w_recip, w_pow2); break;
         case 3: launch_decode<3>(c, W, tab, out, st, w_recip, w_pow2); break;
         case 4: launch_decode<4>(c, W, tab, out, st, w_recip, w_pow2); break;

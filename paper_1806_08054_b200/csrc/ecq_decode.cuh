@@ -99,4 +99,232 @@ decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
     }
 }
 
+
+// ===========================================================================
+// Tiled path.  Every warp works on its own: a tile is 1024 outputs, one run of
+// 32 consecutive entries ("row") per lane, whose codes are R whole words.
+//   * the code words of (tile, worker) -- R*128 contiguous bytes -- are copied
+//     into a warp-private ring with 16-byte asynchronous copies, kRing-1 units
+//     ahead, so that global loads are coalesced and plentiful while each lane
+//     reads its own R words from shared memory without bank conflicts;
+//   * the level steps a_w = scale_w / s of the lane's bucket are loaded one
+//     tile ahead, one worker per lane, and broadcast by shuffles;
+//   * each code is turned into a float without a shift or a conversion where
+//     its bit field allows it: (word & field) | 0x4B000000 is 2^23 + c*2^p, so
+//     one add gives (c - s)*2^p exactly; the power of two is carried through
+//     the sum (a_w is pre-scaled by 2^-22, exact) and undone once per output,
+//     so the terms are summed in ascending w exactly as Eq. 4 is written out;
+//     the subtract and the multiply-add run as packed fp32x2 instructions, two
+//     outputs at a time;
+//   * the 32x32 block of means goes through a swizzled staging buffer so that
+//     the stores to `out` are fully coalesced.
+// ===========================================================================
+constexpr int kDecTileElems = 1024;
+constexpr int kDecWarps = 8;
+constexpr int kDecAreg = 8;                 // level steps loaded per lane and tile
+
+template <int R> struct DecodeTiled {
+    static constexpr int kRing = (R <= 3) ? 16 : (R <= 8 ? 8 : 6);
+    static constexpr int kUnitBytes = R * 128;
+    static constexpr int kFit = (23 / R) & ~1;   // whole fields below bit 23 of a word, even
+    static constexpr int kATabBytes = kDecAreg * 32 * 4;          // a_w per (lane group, worker)
+    static constexpr int kWarpBytes = kRing * kUnitBytes + 4096 + kATabBytes;
+    static constexpr int kSmem = kDecWarps * kWarpBytes;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() {
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <int R>
+__global__ void __launch_bounds__(kDecWarps * 32)
+decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
+                    float* __restrict__ out, const uint32_t n_tiles, const uint64_t n_words,
+                    const float w_recip, const int w_pow2) {
+    using L = DecodeTiled<R>;
+    constexpr int D = L::kRing;
+    constexpr int FIT = L::kFit;
+    constexpr uint32_t mask = (1u << R) - 1u;
+    extern __shared__ __align__(128) uint8_t dsm[];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    uint8_t* const ring = dsm + warp * L::kWarpBytes;
+    uint8_t* const stage = ring + D * L::kUnitBytes;
+    float* const a_tab = reinterpret_cast<float*>(stage + 4096);
+    const uint32_t ring_u32 = smem_u32(ring);
+
+    const uint32_t n_warps = gridDim.x * kDecWarps;
+    const uint32_t gw = blockIdx.x * kDecWarps + warp;
+    const uint32_t my_tiles = gw < n_tiles ? (n_tiles - gw + n_warps - 1) / n_warps : 0;
+    const uint64_t n_units = (uint64_t)my_tiles * W;
+
+    // lanes that share a bucket: gsz consecutive lanes (all 32 above 1024 entries);
+    // a_tab holds, per group of lanes, a_w for w < W (W <= kDecAreg * gsz)
+    const uint32_t gsz = P.bucket >= 1024u ? 32u : (P.bucket >> 5);
+    const uint32_t gl = lane & (gsz - 1);
+    const uint32_t bucket_shift = 31 - __clz(P.bucket);           // bucket is a power of two
+    const uint32_t n_slots = (W + gsz - 1) / gsz;                   // <= kDecAreg
+    float* const a_mine = a_tab + (lane / gsz) * (kDecAreg * gsz);
+
+    // 2^23 + s * 2^(iR): subtracting it from (field | 0x4B000000) leaves (c - s) * 2^(iR)
+    uint64_t T2[FIT / 2];
+#pragma unroll
+    for (int i = 0; i < FIT; i += 2)
+        T2[i / 2] = pack2(__fmaf_rn(P.sf, (float)(1u << (i * R)), 8388608.f),
+                          __fmaf_rn(P.sf, (float)(1u << ((i + 1) * R)), 8388608.f));
+
+    // ---- asynchronous copy of unit n = (tile index n / W, worker n % W) ----
+    uint32_t cp_tile = gw, cp_w = 0, cp_slot = 0;
+    uint64_t cp_unit = 0;
+    auto issue_unit = [&]() {
+        if (cp_unit < n_units) {
+            const uint32_t* src = tab.codes[cp_w] + (uint64_t)cp_tile * (R * 32);
+            const uint32_t dst = ring_u32 + cp_slot;
+#pragma unroll
+            for (int p = 0; p < (8 * R + 31) / 32; ++p) {
+                const int piece = p * 32 + lane;
+                if (piece < 8 * R) cp_async16(dst + piece * 16, src + piece * 4);
+            }
+            if (++cp_w == W) { cp_w = 0; cp_tile += n_warps; }
+            ++cp_unit;
+            cp_slot += L::kUnitBytes;
+            if (cp_slot == D * L::kUnitBytes) cp_slot = 0;
+        }
+        cp_async_commit();
+    };
+    // ---- scales of my bucket for one tile: worker k*gsz + gl in slot k ----
+    auto load_scales = [&](uint32_t tile, float (&dst)[kDecAreg]) {
+        const uint64_t b = ((uint64_t)tile * kDecTileElems + (uint32_t)lane * 32) >> bucket_shift;
+#pragma unroll
+        for (int k = 0; k < kDecAreg; ++k) {
+            if (k < (int)n_slots) {
+                const uint32_t w = k * gsz + gl;
+                dst[k] = (w < W) ? __ldg(tab.scales[w] + b) : 0.f;
+            }
+        }
+    };
+
+#pragma unroll 1
+    for (int i = 0; i < D - 1; ++i) issue_unit();
+    float nxt[kDecAreg];
+    if (my_tiles) load_scales(gw, nxt);
+
+    uint32_t rd_slot = 0;
+    for (uint32_t ti = 0; ti < my_tiles; ++ti) {
+        const uint32_t tile = gw + ti * n_warps;
+        // a_w = scale_w / s, pre-scaled by 2^-22 (exact; only scales below 2^-104 lose
+        // bits, far under the absolute tolerance) against the 2^(iR) of the fields
+#pragma unroll
+        for (int k = 0; k < kDecAreg; ++k)
+            if (k < (int)n_slots)
+                a_mine[k * gsz + gl] = __fmul_rn(__fdiv_rn(nxt[k], P.sf), 0x1p-22f);
+        __syncwarp();
+        if (ti + 1 < my_tiles) load_scales(tile + n_warps, nxt);
+
+        uint64_t acc2[16];                      // outputs (2k, 2k+1) as fp32 pairs
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc2[j] = 0ull;
+
+#pragma unroll 1
+        for (uint32_t w = 0; w < W; ++w) {
+            issue_unit();                       // kRing-1 units ahead, into the slot freed last
+            cp_async_wait<D - 1>();
+            __syncwarp();
+            const float a = a_mine[w];
+            const uint64_t a2 = pack2(a, a);
+            const uint32_t* cwp = reinterpret_cast<const uint32_t*>(ring + rd_slot) + lane * R;
+            uint32_t cw[R + 1];
+            if constexpr (R % 4 == 0) {
+#pragma unroll
+                for (int q = 0; q < R / 4; ++q) {
+                    const uint4 v = reinterpret_cast<const uint4*>(cwp)[q];
+                    cw[4 * q] = v.x; cw[4 * q + 1] = v.y; cw[4 * q + 2] = v.z; cw[4 * q + 3] = v.w;
+                }
+            } else if constexpr (R % 2 == 0) {
+#pragma unroll
+                for (int q = 0; q < R / 2; ++q) {
+                    const uint2 v = reinterpret_cast<const uint2*>(cwp)[q];
+                    cw[2 * q] = v.x; cw[2 * q + 1] = v.y;
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < R; ++q) cw[q] = cwp[q];
+            }
+            cw[R] = 0u;
+            // groups of FIT consecutive codes: one funnel shift brings the group's first
+            // field to bit 0, then every field lies below bit 23
+#pragma unroll
+            for (int j0 = 0; j0 < 32; j0 += FIT) {
+                const int bit = j0 * R, wi = bit >> 5, sh = bit & 31;
+                const uint32_t word = (sh == 0) ? cw[wi]
+                                    : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cw[wi] >> sh)
+                                    : __funnelshift_r(cw[wi], cw[wi + 1], sh);
+#pragma unroll
+                for (int i = 0; i < FIT && j0 + i < 32; i += 2) {
+                    const float F0 = __uint_as_float((word & (mask << (i * R))) | 0x4B000000u);
+                    const float F1 = __uint_as_float((word & (mask << ((i + 1) * R))) | 0x4B000000u);
+                    // (c - s) 2^(iR) a, two outputs per instruction
+                    acc2[(j0 + i) / 2] = fma2(sub2(pack2(F0, F1), T2[i / 2]), a2, acc2[(j0 + i) / 2]);
+                }
+            }
+            __syncwarp();                        // the slot may be overwritten by the next copy
+            rd_slot += L::kUnitBytes;
+            if (rd_slot == D * L::kUnitBytes) rd_slot = 0;
+        }
+
+        // undo the powers of two, divide by W
+        float acc[32];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) unpack2(acc2[j], acc[2 * j], acc[2 * j + 1]);
+        if (w_pow2) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                acc[j] = __fmul_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), w_recip);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                acc[j] = __fdiv_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), (float)W);
+        }
+        // transpose through the staging buffer: row-per-lane -> coalesced 16-byte stores
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<float4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) =
+                make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+        __syncwarp();
+        float* o = out + (uint64_t)tile * kDecTileElems;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
+            const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
+            *reinterpret_cast<float4*>(o + idx * 4) = v;
+        }
+        __syncwarp();
+    }
+    cp_async_wait<0>();
+
+    // ragged end (fewer than 1024 outputs): one thread per output
+    const uint64_t tail0 = (uint64_t)n_tiles * kDecTileElems;
+    const float magic = 8388608.f + P.sf;
+    for (uint64_t i = tail0 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < P.d;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t b = i / P.bucket, bit = i * R, wi = bit >> 5;
+        const uint32_t sh = (uint32_t)(bit & 31);
+        float acc1 = 0.f;
+        for (uint32_t w = 0; w < W; ++w) {
+            const float a = __fdiv_rn(__ldg(tab.scales[w] + b), P.sf);
+            const uint32_t lo = __ldg(tab.codes[w] + wi);
+            const uint32_t hi1 = (sh + R > 32 && wi + 1 < n_words) ? __ldg(tab.codes[w] + wi + 1) : 0u;
+            const uint32_t c = __funnelshift_r(lo, hi1, sh) & mask;
+            acc1 = __fmaf_rn(__fsub_rn(__uint_as_float(0x4B000000u | c), magic), a, acc1);
+        }
+        out[i] = w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, (float)W);
+    }
+}
+
 }  // namespace ecq
