@@ -153,6 +153,7 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, float*
     if ((B & (B - 1)) != 0 || n_tiles64 == 0 || n_tiles64 > 0xFFFFFFFFull) return false;
     const uint32_t gsz = B >= 1024 ? 32 : B / 32;
     if (W > (uint32_t)kDecAreg * gsz) return false;
+    if (n_tiles64 * W > 0xFFFFFFFFull) return false;
     static std::once_flag once[16];
     static int occ[16];
     const int dev = c->device & 15;
@@ -171,7 +172,7 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, float*
     const uint32_t want = (n_tiles + kDecWarps - 1) / kDecWarps;
     if (grid > want) grid = want;
     kern<<<grid, kDecWarps * 32, L::kSmem, st>>>(c->P, W, tab, out, n_tiles, c->n_words, w_recip,
-                                                 w_pow2);
+                                                 w_pow2, 0x4B000000u);
     return true;
 }
 

@@ -127,7 +127,7 @@ template <int R> struct DecodeTiled {
     static constexpr int kRing = (R <= 3) ? 16 : (R <= 8 ? 8 : 6);
     static constexpr int kUnitBytes = R * 128;
     static constexpr int kFit = (23 / R) & ~1;   // whole fields below bit 23 of a word, even
-    static constexpr int kATabBytes = kDecAreg * 32 * 4;          // a_w per (lane group, worker)
+    static constexpr int kATabBytes = kDecAreg * 32 * 8;          // (a_w, a_w) per (lane group, worker)
     static constexpr int kWarpBytes = kRing * kUnitBytes + 4096 + kATabBytes;
     static constexpr int kSmem = kDecWarps * kWarpBytes;
 };
@@ -146,7 +146,7 @@ template <int R>
 __global__ void __launch_bounds__(kDecWarps * 32)
 decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
                     float* __restrict__ out, const uint32_t n_tiles, const uint64_t n_words,
-                    const float w_recip, const int w_pow2) {
+                    const float w_recip, const int w_pow2, const uint32_t exp23_bits) {
     using L = DecodeTiled<R>;
     constexpr int D = L::kRing;
     constexpr int FIT = L::kFit;
@@ -156,13 +156,13 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
     const int warp = threadIdx.x >> 5;
     uint8_t* const ring = dsm + warp * L::kWarpBytes;
     uint8_t* const stage = ring + D * L::kUnitBytes;
-    float* const a_tab = reinterpret_cast<float*>(stage + 4096);
+    float2* const a_tab = reinterpret_cast<float2*>(stage + 4096);
     const uint32_t ring_u32 = smem_u32(ring);
 
     const uint32_t n_warps = gridDim.x * kDecWarps;
     const uint32_t gw = blockIdx.x * kDecWarps + warp;
     const uint32_t my_tiles = gw < n_tiles ? (n_tiles - gw + n_warps - 1) / n_warps : 0;
-    const uint64_t n_units = (uint64_t)my_tiles * W;
+    const uint32_t n_units = my_tiles * W;                          // < 2^32: checked by the host
 
     // lanes that share a bucket: gsz consecutive lanes (all 32 above 1024 entries);
     // a_tab holds, per group of lanes, a_w for w < W (W <= kDecAreg * gsz)
@@ -170,7 +170,7 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
     const uint32_t gl = lane & (gsz - 1);
     const uint32_t bucket_shift = 31 - __clz(P.bucket);           // bucket is a power of two
     const uint32_t n_slots = (W + gsz - 1) / gsz;                   // <= kDecAreg
-    float* const a_mine = a_tab + (lane / gsz) * (kDecAreg * gsz);
+    float2* const a_mine = a_tab + (lane / gsz) * (kDecAreg * gsz);
 
     // 2^23 + s * 2^(iR): subtracting it from (field | 0x4B000000) leaves (c - s) * 2^(iR)
     uint64_t T2[FIT / 2];
@@ -179,9 +179,15 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         T2[i / 2] = pack2(__fmaf_rn(P.sf, (float)(1u << (i * R)), 8388608.f),
                           __fmaf_rn(P.sf, (float)(1u << ((i + 1) * R)), 8388608.f));
 
+    // 2^23 exponent bits for both halves, kept in registers so that mask-and-merge is
+    // one logic instruction per field
+    // (exp23_bits = 0x4B000000 arrives as a kernel argument so that it lives in a register:
+    // a logic instruction takes one immediate, and the field mask is it)
+    const uint64_t magic2 = ((uint64_t)exp23_bits << 32) | exp23_bits;
+
     // ---- asynchronous copy of unit n = (tile index n / W, worker n % W) ----
     uint32_t cp_tile = gw, cp_w = 0, cp_slot = 0;
-    uint64_t cp_unit = 0;
+    uint32_t cp_unit = 0;
     auto issue_unit = [&]() {
         if (cp_unit < n_units) {
             const uint32_t* src = tab.codes[cp_w] + (uint64_t)cp_tile * (R * 32);
@@ -222,8 +228,10 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         // bits, far under the absolute tolerance) against the 2^(iR) of the fields
 #pragma unroll
         for (int k = 0; k < kDecAreg; ++k)
-            if (k < (int)n_slots)
-                a_mine[k * gsz + gl] = __fmul_rn(__fdiv_rn(nxt[k], P.sf), 0x1p-22f);
+            if (k < (int)n_slots) {
+                const float a = __fmul_rn(__fdiv_rn(nxt[k], P.sf), 0x1p-22f);
+                a_mine[k * gsz + gl] = make_float2(a, a);
+            }
         __syncwarp();
         if (ti + 1 < my_tiles) load_scales(tile + n_warps, nxt);
 
@@ -233,11 +241,10 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
 
 #pragma unroll 1
         for (uint32_t w = 0; w < W; ++w) {
-            issue_unit();                       // kRing-1 units ahead, into the slot freed last
-            cp_async_wait<D - 1>();
-            __syncwarp();
-            const float a = a_mine[w];
-            const uint64_t a2 = pack2(a, a);
+            cp_async_wait<D - 2>();             // my pieces of this unit have landed
+            __syncwarp();                       // everyone's have; the previous unit is read out
+            issue_unit();                       // kRing-1 units ahead, into the slot just freed
+            const uint64_t a2 = *reinterpret_cast<const uint64_t*>(a_mine + w);   // (a_w, a_w)
             const uint32_t* cwp = reinterpret_cast<const uint32_t*>(ring + rd_slot) + lane * R;
             uint32_t cw[R + 1];
             if constexpr (R % 4 == 0) {
@@ -265,15 +272,16 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
                 const uint32_t word = (sh == 0) ? cw[wi]
                                     : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cw[wi] >> sh)
                                     : __funnelshift_r(cw[wi], cw[wi + 1], sh);
+                // both halves of a 64-bit pair hold the word: one 64-bit and/or then yields
+                // the float bits of two fields side by side, ready for the packed arithmetic
+                const uint64_t w2 = ((uint64_t)word << 32) | word;
 #pragma unroll
                 for (int i = 0; i < FIT && j0 + i < 32; i += 2) {
-                    const float F0 = __uint_as_float((word & (mask << (i * R))) | 0x4B000000u);
-                    const float F1 = __uint_as_float((word & (mask << ((i + 1) * R))) | 0x4B000000u);
+                    const uint64_t m2 = ((uint64_t)(mask << ((i + 1) * R)) << 32) | (uint64_t)(mask << (i * R));
                     // (c - s) 2^(iR) a, two outputs per instruction
-                    acc2[(j0 + i) / 2] = fma2(sub2(pack2(F0, F1), T2[i / 2]), a2, acc2[(j0 + i) / 2]);
+                    acc2[(j0 + i) / 2] = fma2(sub2((w2 & m2) | magic2, T2[i / 2]), a2, acc2[(j0 + i) / 2]);
                 }
             }
-            __syncwarp();                        // the slot may be overwritten by the next copy
             rd_slot += L::kUnitBytes;
             if (rd_slot == D * L::kUnitBytes) rd_slot = 0;
         }
