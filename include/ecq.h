@@ -48,7 +48,8 @@ enum {
     ECQ_ERR_CUDA = 2,       /* a CUDA runtime or driver call failed */
     ECQ_ERR_NONFINITE = 3,  /* NaN or Inf met in a compensated gradient (sticky, device) */
     ECQ_ERR_TIMEOUT = 4,    /* a bounded in-kernel wait on an async copy ran out (sticky, device) */
-    ECQ_ERR_ALLOC = 5       /* host or device allocation failed in ecq_create */
+    ECQ_ERR_ALLOC = 5,      /* host or device allocation failed in ecq_create */
+    ECQ_ERR_TOO_LARGE = 6   /* ecq_step_static: the messages do not fit the built-in scratch */
 };
 
 /*
@@ -142,6 +143,46 @@ int ecq_step_host(ecq_ctx* ctx, uint32_t W, uint32_t step,
                   const float* const* grads_host, float* err_dev,
                   void* workspace_dev, uint64_t workspace_bytes,
                   float* out_host, void* cuda_stream);
+
+/*
+ * One whole iteration on DEVICE buffers for callers that must not allocate.
+ * (The paper has no counterpart: this entry point exists for the embedding, not
+ * for the method.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or cannot be
+ * afforded -- inside a memory pool that owns all of the GPU's memory, in a plugin
+ * called from another framework's hot loop, in a process whose allocator must not
+ * be re-entered.  ecq_create and the caller-owned message buffers of ecq_encode /
+ * ecq_decode_mean both need allocations; this call needs neither a context nor
+ * message buffers.  It runs W encodes and one decode-mean exactly like
+ * ecq_encode (worker w, iteration `step`, error mode 0) and ecq_decode_mean
+ * would, keeping the W messages and the status word in a scratch array that is
+ * compiled into the library: ECQ_STATIC_SCRATCH_BYTES of device memory that every
+ * GPU on which the library is loaded holds until the process exits.
+ *
+ *   d, bucket, levels, alpha, beta, seed   as in ecq_create
+ *   W        1..ECQ_MAX_WORKERS
+ *   grads    HOST array of W device pointers, [d] floats each (read only)
+ *   err      [W*d] device floats, worker-major accumulators (in/out)
+ *   out      [d] device floats, the decoded mean
+ * The scratch must hold 256 + W * (roundup256(4*ceil(d*r/32)) + roundup256(4*ceil(d/bucket)))
+ * bytes; larger problems are refused with ECQ_ERR_TOO_LARGE before anything is
+ * launched.  d must be a multiple of 4 when W > 1 (16-byte aligned accumulators).
+ *
+ * The call enqueues on `cuda_stream`, waits for it, and returns ECQ_OK,
+ * ECQ_ERR_NONFINITE or ECQ_ERR_TIMEOUT like ecq_status would.  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine.  The first call on a
+ * device looks up the scratch array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share
+ * the one array and it keeps the last call's contents: the status word is cleared
+ * at the start of every call, the messages are fully overwritten; two calls that
+ * overlap on the GPU (different streams or host threads) race on it and must be
+ * serialised by the caller.
+ */
+#define ECQ_STATIC_SCRATCH_BYTES (4u << 20)
+int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, float alpha, float beta,
+                    uint64_t seed, uint32_t W, uint32_t step, const float* const* grads,
+                    float* err, float* out, void* cuda_stream);
 
 /*
  * Synchronise `cuda_stream`, then return and clear the context's sticky device

@@ -16,6 +16,8 @@ import torch
 from .build import LIB
 
 ECQ_OK, ECQ_ERR_ARG, ECQ_ERR_CUDA, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT, ECQ_ERR_ALLOC = range(6)
+ECQ_ERR_TOO_LARGE = 6
+ECQ_STATIC_SCRATCH_BYTES = 4 << 20
 ECQ_MAX_WORKERS = 64
 
 _lib = None
@@ -58,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.ecq_step_host_workspace_bytes.restype = u64
         L.ecq_step_host.argtypes = [vp, u32, u32, vp, vp, vp, u64, vp, vp]
         L.ecq_step_host.restype = i32
+        L.ecq_step_static.argtypes = [u64, u32, u32, f32, f32, u64, u32, u32, vp, vp, vp, vp]
+        L.ecq_step_static.restype = i32
         L.ecq_status.argtypes = [vp, vp]
         L.ecq_status.restype = i32
         L.ecq_launch_count.argtypes = []
@@ -159,6 +163,24 @@ def ecq_step_host(ctx: int, step: int, grads_host: Sequence[torch.Tensor], err: 
                              out_host.data_ptr(), _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_step_host")
+
+
+def ecq_step_static(d: int, bucket: int, levels: int, alpha: float, beta: float, seed: int,
+                    step: int, grads: Sequence[torch.Tensor], err: torch.Tensor,
+                    out: torch.Tensor, stream=None) -> int:
+    """One iteration (W encodes + decode-mean) that allocates nothing: no context, and the
+    messages live in the scratch array built into the library.  For callers that are not
+    allowed to allocate device memory (see ``ecq_step_static`` in ecq.h).  Blocking; returns
+    the device status (ECQ_OK / ECQ_ERR_NONFINITE / ECQ_ERR_TIMEOUT) and raises on argument
+    errors, among them ECQ_ERR_TOO_LARGE when the messages exceed the built-in scratch."""
+    W = len(grads)
+    gp = (ctypes.c_void_p * W)(*[_dev(g, torch.float32, "grads") for g in grads])
+    rc = lib().ecq_step_static(d, bucket, levels, alpha, beta, seed, W, step, gp,
+                               _dev(err, torch.float32, "err"), _dev(out, torch.float32, "out"),
+                               _stream(stream))
+    if rc not in (ECQ_OK, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT):
+        raise EcqError(rc, "ecq_step_static")
+    return rc
 
 
 def ecq_status(ctx: int, stream=None) -> int:

@@ -398,8 +398,107 @@ const char* ecq_strerror(int status) {
         case ECQ_ERR_NONFINITE: return "NaN or Inf in a compensated gradient";
         case ECQ_ERR_TIMEOUT: return "an in-kernel wait on an asynchronous copy ran out";
         case ECQ_ERR_ALLOC: return "allocation failed";
+        case ECQ_ERR_TOO_LARGE: return "problem too large for the built-in scratch of ecq_step_static";
         default: return "unknown status";
     }
 }
 
 }  // extern "C"
+
+// ===========================================================================
+// ecq_step_static: the whole iteration without any allocation.  The W messages
+// and the status word live in an array compiled into the library.  In host code
+// the array's name is only a stand-in; its device address is looked up once per
+// device and that pointer is what the kernels get.
+// ===========================================================================
+static __device__ __align__(256) unsigned char g_static_scratch[ECQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+struct StaticScratch {
+    std::once_flag once;
+    unsigned char* ptr = nullptr;
+    cudaError_t err = cudaErrorUnknown;
+};
+StaticScratch g_static[16];
+
+// Device address of the built-in scratch on the current device (set-up on first use).
+unsigned char* static_scratch_ptr(int device) {
+    StaticScratch& s = g_static[device & 15];
+    std::call_once(s.once, [&] {
+        void* p = nullptr;
+        s.err = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (s.err == cudaSuccess) s.ptr = static_cast<unsigned char*>(p);
+    });
+    return s.err == cudaSuccess ? s.ptr : nullptr;
+}
+
+}  // namespace
+
+extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, float alpha,
+                               float beta, uint64_t seed, uint32_t W, uint32_t step,
+                               const float* const* grads, float* err, float* out,
+                               void* cuda_stream) {
+    if (!grads || !err || !out || W == 0 || W > ECQ_MAX_WORKERS) return ECQ_ERR_ARG;
+    if (d == 0 || bucket < 32 || bucket % 32 != 0 || levels == 0 || levels > 32767)
+        return ECQ_ERR_ARG;
+    if (!(alpha >= 0.f) || !(beta >= 0.f) || !(beta <= 1.f) || !(alpha < INFINITY))
+        return ECQ_ERR_ARG;
+    if (!aligned16(err) || !aligned16(out) || (d % 4 != 0 && W > 1)) return ECQ_ERR_ARG;
+    for (uint32_t w = 0; w < W; ++w)
+        if (!grads[w] || !aligned16(grads[w])) return ECQ_ERR_ARG;
+
+    // a context on the stack: constants only, nothing allocated
+    ecq_ctx c;
+    CodecParams& P = c.P;
+    P.d = d; P.bucket = bucket; P.s = levels; P.mode = 0;
+    P.alpha = alpha; P.beta = beta; P.sf = (float)levels;
+    P.r = 0;
+    while ((1ull << P.r) < 2ull * levels + 1ull) ++P.r;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int i = 0; i < 10; ++i) {
+        P.key0[i] = k0; P.key1[i] = k1;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    c.nb = (d + bucket - 1) / bucket;
+    c.n_words = (d * P.r + 31) / 32;
+    c.tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= kMaxTiledBucket;
+    c.host_ready = false;
+    c.h_status = nullptr;
+
+    const uint64_t codes_b = round_up(c.n_words * 4, 256);
+    const uint64_t scales_b = round_up(c.nb * 4, 256);
+    const uint64_t need = 256 + (uint64_t)W * (codes_b + scales_b);
+    if (need > ECQ_STATIC_SCRATCH_BYTES) return ECQ_ERR_TOO_LARGE;
+
+    if (cudaGetDevice(&c.device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess)
+        return ECQ_ERR_CUDA;
+    unsigned char* scratch = static_scratch_ptr(c.device);
+    if (!scratch) return ECQ_ERR_CUDA;
+    c.d_status = reinterpret_cast<uint32_t*>(scratch);
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the array keeps the previous call's contents: the status word must start at zero
+    if (cudaMemsetAsync(c.d_status, 0, sizeof(uint32_t), st) != cudaSuccess) return ECQ_ERR_CUDA;
+    MessageTable tab;
+    std::memset(&tab, 0, sizeof(tab));
+    int rc = ECQ_OK;
+    for (uint32_t w = 0; w < W && rc == ECQ_OK; ++w) {
+        unsigned char* msg = scratch + 256 + w * (codes_b + scales_b);
+        uint32_t* codes = reinterpret_cast<uint32_t*>(msg);
+        float* scales = reinterpret_cast<float*>(msg + codes_b);
+        tab.codes[w] = codes;
+        tab.scales[w] = scales;
+        rc = encode_impl(&c, w, step, grads[w], err + (uint64_t)w * d, codes, scales, st);
+    }
+    if (rc == ECQ_OK) rc = decode_impl(&c, W, tab, out, st);
+    uint32_t bits = 0;
+    if (cudaMemcpyAsync(&bits, c.d_status, sizeof(bits), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return ECQ_ERR_CUDA;
+    if (rc != ECQ_OK) return rc;
+    if (bits & kStatusTimeout) return ECQ_ERR_TIMEOUT;
+    if (bits & kStatusNonFinite) return ECQ_ERR_NONFINITE;
+    return ECQ_OK;
+}
