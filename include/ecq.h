@@ -42,6 +42,8 @@ extern "C" {
 
 typedef struct ecq_ctx ecq_ctx;
 
+#define ECQ_MAX_WORKERS 64   /* most workers one batched or receiver-side call takes */
+
 enum {
     ECQ_OK = 0,
     ECQ_ERR_ARG = 1,        /* null / misaligned pointer, size or range violation */
@@ -112,6 +114,21 @@ int ecq_encode(ecq_ctx* ctx, uint32_t worker, uint32_t step, const float* grad,
                float* err, uint32_t* codes, float* scales, void* cuda_stream);
 
 /*
+ * ecq_encode for workers 0..W-1 of one iteration in ONE kernel launch (Algorithm 1,
+ * the loop "for p = 1..P" of phase 1, on a single GPU that holds all P workers'
+ * slices).  Results are identical to W calls of ecq_encode(ctx, w, step, grads[w],
+ * errs[w], codes[w], scales[w]); a single launch spares W-1 launch ramps and tails,
+ * which matters for vectors of tens of megabytes.
+ *   W       1..ECQ_MAX_WORKERS
+ *   grads, errs, codes, scales   HOST arrays of W device pointers each, with the
+ *           meaning, sizes and alignment of ecq_encode's arguments; read before the
+ *           call returns
+ */
+int ecq_encode_batch(ecq_ctx* ctx, uint32_t W, uint32_t step, const float* const* grads,
+                     float* const* errs, uint32_t* const* codes, float* const* scales,
+                     void* cuda_stream);
+
+/*
  * Receiver side (Eq. 4 and Algorithm 1, "compute global gradients"):
  *   out_i = (1/W) * sum_{w<W} q_{w,i} * (scales_w[b(i)] / s)
  *   W       number of messages, 1..ECQ_MAX_WORKERS
@@ -120,7 +137,6 @@ int ecq_encode(ecq_ctx* ctx, uint32_t worker, uint32_t step, const float* grad,
  *   out [d] the averaged dequantised gradient
  * The two pointer arrays are read before the call returns.
  */
-#define ECQ_MAX_WORKERS 64
 int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
                     const float* const* scales, float* out, void* cuda_stream);
 

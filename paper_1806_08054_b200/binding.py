@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.ecq_codes_words.restype = u64
         L.ecq_encode.argtypes = [vp, u32, u32, vp, vp, vp, vp, vp]
         L.ecq_encode.restype = i32
+        L.ecq_encode_batch.argtypes = [vp, u32, u32, vp, vp, vp, vp, vp]
+        L.ecq_encode_batch.restype = i32
         L.ecq_decode_mean.argtypes = [vp, u32, vp, vp, vp, vp]
         L.ecq_decode_mean.restype = i32
         L.ecq_step_host_workspace_bytes.argtypes = [vp, u32]
@@ -129,6 +131,21 @@ def ecq_encode(ctx: int, worker: int, step: int, grad: torch.Tensor, err: torch.
                           _dev(scales, torch.float32, "scales"), _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_encode")
+
+
+def ecq_encode_batch(ctx: int, step: int, grads: Sequence[torch.Tensor],
+                     errs: Sequence[torch.Tensor], codes: Sequence[torch.Tensor],
+                     scales: Sequence[torch.Tensor], stream=None) -> None:
+    """Enqueue the sender-side kernel for workers 0..len(grads)-1 as one launch."""
+    W = len(grads)
+    if not (len(errs) == len(codes) == len(scales) == W):
+        raise ValueError("grads, errs, codes and scales must have one entry per worker")
+    arr = lambda ts, dt, nm: (ctypes.c_void_p * W)(*[_dev(x, dt, nm) for x in ts])  # noqa: E731
+    rc = lib().ecq_encode_batch(ctx, W, step, arr(grads, torch.float32, "grads"),
+                                arr(errs, torch.float32, "errs"), arr(codes, torch.int32, "codes"),
+                                arr(scales, torch.float32, "scales"), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_encode_batch")
 
 
 def ecq_decode_mean(ctx: int, codes: Sequence[torch.Tensor], scales: Sequence[torch.Tensor],

@@ -74,14 +74,22 @@ bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
            CUDA_SUCCESS;
 }
 
-template <int R>
-int launch_encode_tiled(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
-                        uint32_t* codes, float* scales, cudaStream_t st, uint32_t n_tiles) {
+// Buffers of one batch entry as the launchers see them.
+struct WorkerBuffers {
+    const float* g;
+    float* h;
+    uint32_t* codes;
+    float* scales;
+};
+
+template <int R, bool MODE1>
+int launch_encode_tiled(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
+                        const WorkerBuffers* wb, cudaStream_t st, uint32_t n_tiles) {
     using L = EncodeSmem<R>;
     static std::once_flag once[16];
     static int occ[16];
     const int dev = c->device & 15;
-    auto kern = encode_tiled_kernel<R>;
+    auto kern = encode_tiled_kernel<R, MODE1>;
     std::call_once(once[dev], [&] {
         int o = 0;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) ==
@@ -91,15 +99,34 @@ int launch_encode_tiled(ecq_ctx* c, uint32_t worker, uint32_t step, const float*
             occ[dev] = o;
     });
     if (occ[dev] <= 0) return ECQ_ERR_CUDA;
-    CUtensorMap tm_g, tm_h;
+    EncodeBatch bt;
     const uint64_t rows = (uint64_t)n_tiles * kTileRows;
-    if (!make_tile_map(&tm_g, g, rows) || !make_tile_map(&tm_h, h, rows)) return ECQ_ERR_CUDA;
+    for (uint32_t e = 0; e < (uint32_t)kMaxBatch; ++e) {
+        const uint32_t src = e < n_workers ? e : 0;       // unused entries repeat entry 0
+        if (e < n_workers) {
+            if (!make_tile_map(&bt.tm_g[e], wb[e].g, rows) || !make_tile_map(&bt.tm_h[e], wb[e].h, rows))
+                return ECQ_ERR_CUDA;
+        } else {
+            bt.tm_g[e] = bt.tm_g[0];
+            bt.tm_h[e] = bt.tm_h[0];
+        }
+        bt.g[e] = wb[src].g; bt.h[e] = wb[src].h;
+        bt.codes[e] = wb[src].codes; bt.scales[e] = wb[src].scales;
+    }
+    const uint64_t total = (uint64_t)n_tiles * n_workers;
     uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
-    if (grid > n_tiles) grid = n_tiles;
-    kern<<<grid, kEncodeThreads, L::kTotal, st>>>(tm_g, tm_h, c->P, worker, step, g, h, codes,
-                                                  scales, c->d_status, n_tiles);
+    if (grid > total) grid = (uint32_t)total;
+    kern<<<grid, kEncodeThreads, L::kTotal, st>>>(bt, c->P, worker_base, n_workers, step,
+                                                  c->d_status, n_tiles);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+template <int R>
+int launch_encode_tiled_mode(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
+                             const WorkerBuffers* wb, cudaStream_t st, uint32_t n_tiles) {
+    return c->P.mode ? launch_encode_tiled<R, true>(c, worker_base, n_workers, step, wb, st, n_tiles)
+                     : launch_encode_tiled<R, false>(c, worker_base, n_workers, step, wb, st, n_tiles);
 }
 
 int launch_encode_generic(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
@@ -112,23 +139,37 @@ int launch_encode_generic(ecq_ctx* c, uint32_t worker, uint32_t step, const floa
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
 }
 
-int encode_impl(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
-                uint32_t* codes, float* scales, cudaStream_t st) {
-    const uint32_t n_tiles = c->tiled_ok ? (uint32_t)(c->P.d / kTileElems) : 0;
-    if (n_tiles > 0) {
+// Encode n_workers vectors (workers worker_base .. worker_base + n_workers - 1).  The tiled
+// path takes the whole batch in one launch; other shapes go one launch per worker.
+int encode_batch_impl(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
+                      const WorkerBuffers* wb, cudaStream_t st) {
+    const uint64_t n_tiles64 = c->tiled_ok ? c->P.d / kTileElems : 0;
+    if (n_tiles64 > 0 && n_tiles64 * n_workers <= 0xFFFFFFFFull && n_tiles64 * kTileRows <= 0x7FFFFFFFull) {
+        const uint32_t n_tiles = (uint32_t)n_tiles64;
         switch (c->P.r) {
-            case 2: return launch_encode_tiled<2>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 3: return launch_encode_tiled<3>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 4: return launch_encode_tiled<4>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 5: return launch_encode_tiled<5>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 6: return launch_encode_tiled<6>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 7: return launch_encode_tiled<7>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 8: return launch_encode_tiled<8>(c, worker, step, g, h, codes, scales, st, n_tiles);
-            case 9: return launch_encode_tiled<9>(c, worker, step, g, h, codes, scales, st, n_tiles);
+            case 2: return launch_encode_tiled_mode<2>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 3: return launch_encode_tiled_mode<3>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 4: return launch_encode_tiled_mode<4>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 5: return launch_encode_tiled_mode<5>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 6: return launch_encode_tiled_mode<6>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 7: return launch_encode_tiled_mode<7>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 8: return launch_encode_tiled_mode<8>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 9: return launch_encode_tiled_mode<9>(c, worker_base, n_workers, step, wb, st, n_tiles);
             default: break;
         }
     }
-    return launch_encode_generic(c, worker, step, g, h, codes, scales, st);
+    for (uint32_t e = 0; e < n_workers; ++e) {
+        const int rc = launch_encode_generic(c, worker_base + e, step, wb[e].g, wb[e].h, wb[e].codes,
+                                             wb[e].scales, st);
+        if (rc != ECQ_OK) return rc;
+    }
+    return ECQ_OK;
+}
+
+int encode_impl(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
+                uint32_t* codes, float* scales, cudaStream_t st) {
+    const WorkerBuffers wb = {g, h, codes, scales};
+    return encode_batch_impl(c, worker, 1, step, &wb, st);
 }
 
 template <int R>
@@ -289,6 +330,21 @@ int ecq_encode(ecq_ctx* c, uint32_t worker, uint32_t step, const float* grad, fl
         return ECQ_ERR_ARG;
     return encode_impl(c, worker, step, grad, err, codes, scales,
                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ecq_encode_batch(ecq_ctx* c, uint32_t W, uint32_t step, const float* const* grads,
+                     float* const* errs, uint32_t* const* codes, float* const* scales,
+                     void* cuda_stream) {
+    if (!c || !grads || !errs || !codes || !scales || W == 0 || W > ECQ_MAX_WORKERS)
+        return ECQ_ERR_ARG;
+    WorkerBuffers wb[ECQ_MAX_WORKERS];
+    for (uint32_t w = 0; w < W; ++w) {
+        if (!grads[w] || !errs[w] || !codes[w] || !scales[w]) return ECQ_ERR_ARG;
+        if (!aligned16(grads[w]) || !aligned16(errs[w]) || !aligned16(codes[w]) || !aligned4(scales[w]))
+            return ECQ_ERR_ARG;
+        wb[w] = {grads[w], errs[w], codes[w], scales[w]};
+    }
+    return encode_batch_impl(c, 0, W, step, wb, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int ecq_decode_mean(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,

@@ -160,12 +160,24 @@ __device__ __forceinline__ float max3_abs_nan(float m, float a, float b) {
     return r;
 }
 
-template <int R>
+// The buffers of the workers that one launch serves (a batch may hold one worker).
+constexpr int kMaxBatch = 64;
+struct alignas(64) EncodeBatch {
+    CUtensorMap tm_g[kMaxBatch];    // tiled views of grad (loads)
+    CUtensorMap tm_h[kMaxBatch];    // tiled views of err (loads and stores)
+    const float* g[kMaxBatch];
+    float* h[kMaxBatch];
+    uint32_t* codes[kMaxBatch];
+    float* scales[kMaxBatch];
+};
+
+// One launch walks the tiles of n_workers vectors: global tile T is tile T % n_tiles
+// of batch entry T / n_tiles, whose Philox stream is that of worker worker_base + entry.
+template <int R, bool MODE1>
 __global__ void __launch_bounds__(kEncodeThreads, kEncodeCtasPerSm)
-encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_h,
-                    const CodecParams P, const uint32_t worker, const uint32_t step,
-                    const float* __restrict__ g, float* h, uint32_t* __restrict__ codes,
-                    float* __restrict__ scales, uint32_t* status, const uint32_t n_tiles) {
+encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
+                    const uint32_t worker_base, const uint32_t n_workers, const uint32_t step,
+                    uint32_t* status, const uint32_t n_tiles) {
     using L = EncodeSmem<R>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -177,16 +189,18 @@ encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    auto issue_load = [&](uint32_t tile) {
+    const uint32_t total_tiles = n_workers * n_tiles;       // < 2^32: checked by the host
+    auto issue_load = [&](uint32_t T) {
+        const uint32_t e = T / n_tiles, tile = T - e * n_tiles;
         mbar_arrive_expect_tx(bar_full, 2 * kTileBytes);
-        tma_load_2d(base + L::kLoadOff, &tm_g, 0, (int)(tile * kTileRows), bar_full);
-        tma_load_2d(base + L::kLoadOff + kTileBytes, &tm_h, 0, (int)(tile * kTileRows), bar_full);
+        tma_load_2d(base + L::kLoadOff, &bt.tm_g[e], 0, (int)(tile * kTileRows), bar_full);
+        tma_load_2d(base + L::kLoadOff + kTileBytes, &bt.tm_h[e], 0, (int)(tile * kTileRows), bar_full);
     };
     if (tid == 0) {
         mbar_init(bar_full, 1);
         *s_abort = 0;
         fence_mbar_init();
-        if (blockIdx.x < n_tiles) issue_load(blockIdx.x);
+        if (blockIdx.x < total_tiles) issue_load(blockIdx.x);
     }
     __syncthreads();
 
@@ -194,13 +208,18 @@ encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     const uint32_t rpb = P.bucket >> 5;                    // rows per bucket, power of two <= 128
     const uint32_t buckets_per_tile = kTileElems / P.bucket;
     const float magic_code = 12582912.f + P.sf;            // 1.5*2^23 + s, exact
+    const uint64_t magic2 = pack2(magic_code, magic_code);
+    const uint64_t alpha2 = pack2(P.alpha, P.alpha), beta2 = pack2(P.beta, P.beta);
+    const uint64_t two23_2 = pack2(8388608.f, 8388608.f), ulp24_2 = pack2(0x1p-24f, 0x1p-24f);
     const uint8_t* const g_row = sm + L::kLoadOff + tid * 128;
     const uint8_t* const h_row = g_row + kTileBytes;
     uint8_t* const hout_row = sm + L::kHoutOff + tid * 128;
     uint32_t* const cout_row = reinterpret_cast<uint32_t*>(sm + L::kCoutOff) + tid * R;
 
     uint32_t parity = 0;
-    for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, parity ^= 1u) {
+    for (uint32_t T = blockIdx.x; T < total_tiles; T += gridDim.x, parity ^= 1u) {
+        const uint32_t entry = T / n_tiles, tile = T - entry * n_tiles;
+        const uint32_t worker = worker_base + entry;
         if (!mbar_wait(bar_full, parity)) { *s_abort = 1; atomicOr(status, kStatusTimeout); }
 
         // my row of g and h -> registers
@@ -215,85 +234,121 @@ encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
         float mf = 0.f;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            mf = max3_abs_nan(mf, __fmaf_rn(P.alpha, H[c].x, G[c].x), __fmaf_rn(P.alpha, H[c].y, G[c].y));
-            mf = max3_abs_nan(mf, __fmaf_rn(P.alpha, H[c].z, G[c].z), __fmaf_rn(P.alpha, H[c].w, G[c].w));
+            float v0, v1, v2, v3;
+            unpack2(fma2(alpha2, pack2(H[c].x, H[c].y), pack2(G[c].x, G[c].y)), v0, v1);
+            unpack2(fma2(alpha2, pack2(H[c].z, H[c].w), pack2(G[c].z, G[c].w)), v2, v3);
+            mf = max3_abs_nan(mf, v0, v1);
+            mf = max3_abs_nan(mf, v2, v3);
         }
         // non-negative floats and NaN (0x7FFFFFFF) order like their bit patterns
         uint32_t m = __float_as_uint(mf) & 0x7FFFFFFFu;
         for (uint32_t o = 1; o < rpb && o < 32; o <<= 1)
             m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
         if (rpb > 32 && lane == 0) s_wmax[warp] = m;
-        // the stores of the previous tile must have read the staging buffer
-        if (tid == 0) bulk_wait_read0();
-        __syncthreads();                                   // load buffer and staging are free
+        __syncthreads();                                   // the load buffer is free
         if (*s_abort) break;                               // uniform: set before the barrier
-        if (tid == 0 && tile + gridDim.x < n_tiles) issue_load(tile + gridDim.x);
+        if (tid == 0 && T + gridDim.x < total_tiles) issue_load(T + gridDim.x);
         if (rpb == 64) m = max(s_wmax[warp & ~1], s_wmax[warp | 1]);
         if (rpb == 128) m = max(max(s_wmax[0], s_wmax[1]), max(s_wmax[2], s_wmax[3]));
         const BucketScale bs = bucket_scale(m, P.sf);
         if ((tid & (rpb - 1)) == 0) {
-            scales[(uint64_t)tile * buckets_per_tile + tid / rpb] = bs.scale;
+            bt.scales[entry][(uint64_t)tile * buckets_per_tile + tid / rpb] = bs.scale;
             if (bs.kind == 2) atomicOr(status, kStatusNonFinite);
         }
 
-        // round, new h (kept in H), pack 32 codes into R words.  The codes enter a
-        // 64-bit window as (float bits of q + s + 1.5*2^23) << pos; the constant
-        // high bits are removed once per output word.
+        // round, new h (written over H), pack 32 codes into R words.  The codes enter
+        // a 64-bit window as (float bits of q + s + 1.5*2^23) << pos; the constant high
+        // bits are removed once per output word.  The fp32 steps run as packed fp32x2
+        // instructions on two neighbouring entries (each half is the same IEEE
+        // operation as in the scalar form).
         const uint64_t blk0 = (uint64_t)tile * (kTileElems / 4) + (uint32_t)tid * 8;
         uint32_t wout[R];
         uint64_t acc = 0, junk = 0;
         int nbits = 0, kw = 0;
+        if (bs.kind == 0) {
+            const uint64_t inv2 = pack2(bs.inv, bs.inv);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const float gv[4] = {G[c].x, G[c].y, G[c].z, G[c].w};
-            const float hv[4] = {H[c].x, H[c].y, H[c].z, H[c].w};
-            float hn[4];
-            uint32_t cb[4];
-            if (bs.kind == 0) {
+            for (int c = 0; c < 8; ++c) {
                 uint32_t Rw[4];
                 const uint64_t blk = blk0 + c;
                 philox4x32_10(P, (uint32_t)blk, (uint32_t)(blk >> 32), worker, step, Rw);
+                uint32_t cb[4];
+                float hn[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float v = __fmaf_rn(P.alpha, hv[j], gv[j]);
-                    const uint32_t sgn = __float_as_uint(v) & 0x80000000u;
-                    const float x = fminf(__fmul_rn(fabsf(v), bs.inv), P.sf);
-                    const float lf = __fsub_rn(__fadd_rz(x, 8388608.f), 8388608.f);   // floor
-                    const float f = __fsub_rn(x, lf);
-                    const float u = __fmul_rn(__uint2float_rn(Rw[j] >> 8), 0x1p-24f);
-                    const float mlev = __fadd_rn(lf, (u < f) ? 1.f : 0.f);
+                for (int hlf = 0; hlf < 2; ++hlf) {
+                    const uint64_t g2 = hlf ? pack2(G[c].z, G[c].w) : pack2(G[c].x, G[c].y);
+                    const uint64_t h2 = hlf ? pack2(H[c].z, H[c].w) : pack2(H[c].x, H[c].y);
+                    const uint64_t v2 = fma2(alpha2, h2, g2);                       // Eq. 7
+                    const uint64_t sgn2 = v2 & 0x8000000080000000ull;
+                    float xs0, xs1;
+                    unpack2(mul2(v2, inv2), xs0, xs1);                              // |v| s/scale, signed
+                    const uint64_t x2 = pack2(fminf(fabsf(xs0), P.sf), fminf(fabsf(xs1), P.sf));
+                    const uint64_t lf2 = sub2(add2_rz(x2, two23_2), two23_2);       // floor
+                    float f0, f1, u0, u1;
+                    unpack2(sub2(x2, lf2), f0, f1);
+                    unpack2(mul2(pack2(__uint2float_rn(Rw[2 * hlf] >> 8),
+                                       __uint2float_rn(Rw[2 * hlf + 1] >> 8)), ulp24_2), u0, u1);
+                    const uint64_t m2 = add2(lf2, pack2((u0 < f0) ? 1.f : 0.f, (u1 < f1) ? 1.f : 0.f));
                     // work on sgn(v)*g so that the level stays non-negative: negation
                     // commutes with rounding, and a zero level leaves g untouched
-                    const float gsn = __uint_as_float(__float_as_uint(P.mode ? v : gv[j]) ^ sgn);
-                    const float esn = __fsub_rn(gsn, __fmul_rn(mlev, bs.a));
-                    const float e = __uint_as_float(__float_as_uint(esn) ^ sgn);
-                    hn[j] = __fmaf_rn(P.beta, hv[j], e);
-                    const float q = __uint_as_float(__float_as_uint(mlev) ^ sgn);
-                    cb[j] = __float_as_uint(__fadd_rn(q, magic_code));     // 0x4B400000 + q + s
+                    const uint64_t gsn2 = (MODE1 ? v2 : g2) ^ sgn2;
+                    // (the product stays scalar: ptxas contracts a packed multiply with a
+                    // following packed subtract into one fused operation, which would drop
+                    // the rounding of g~ that Eq. 6 books)
+                    float m0, m1;
+                    unpack2(m2, m0, m1);
+                    const uint64_t e2 = sub2(gsn2, pack2(__fmul_rn(m0, bs.a), __fmul_rn(m1, bs.a))) ^ sgn2;
+                    unpack2(fma2(beta2, h2, e2), hn[2 * hlf], hn[2 * hlf + 1]);     // Eq. 6
+                    const uint64_t c2 = add2(m2 ^ sgn2, magic2);                    // 0x4B400000 + q + s
+                    cb[2 * hlf] = (uint32_t)c2;
+                    cb[2 * hlf + 1] = (uint32_t)(c2 >> 32);
                 }
-            } else {
+                H[c] = make_float4(hn[0], hn[1], hn[2], hn[3]);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const float v = __fmaf_rn(P.alpha, hv[j], gv[j]);
-                    cb[j] = 0x4B400000u + P.s;
-                    hn[j] = (bs.kind == 1) ? __fmaf_rn(P.beta, hv[j], P.mode ? v : gv[j]) : hv[j];
+                    acc += (uint64_t)cb[j] * (uint64_t)(1u << nbits);
+                    junk += (uint64_t)0x4B400000u << nbits;
+                    nbits += R;
+                    if (nbits >= 32) {
+                        acc -= junk; junk = 0;
+                        wout[kw++] = (uint32_t)acc;
+                        acc >>= 32;
+                        nbits -= 32;
+                    }
                 }
             }
-            *reinterpret_cast<float4*>(hout_row + (((uint32_t)c << 4) ^ sw)) =
-                make_float4(hn[0], hn[1], hn[2], hn[3]);
+        } else {
+            // all levels zero (code s): an all-zero bucket books beta*h + g, a non-finite one
+            // keeps h
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                acc += (uint64_t)cb[j] * (uint64_t)(1u << nbits);
-                junk += (uint64_t)0x4B400000u << nbits;
-                nbits += R;
-                if (nbits >= 32) {
-                    acc -= junk; junk = 0;
-                    wout[kw++] = (uint32_t)acc;
-                    acc >>= 32;
-                    nbits -= 32;
+            for (int c = 0; c < 8; ++c) {
+                if (bs.kind == 1) {
+                    const float gv[4] = {G[c].x, G[c].y, G[c].z, G[c].w};
+                    const float hv[4] = {H[c].x, H[c].y, H[c].z, H[c].w};
+                    float hn[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        hn[j] = __fmaf_rn(P.beta, hv[j], MODE1 ? __fmaf_rn(P.alpha, hv[j], gv[j]) : gv[j]);
+                    H[c] = make_float4(hn[0], hn[1], hn[2], hn[3]);
                 }
+            }
+            uint64_t zacc = 0;
+            int zbits = 0, zk = 0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                zacc |= (uint64_t)P.s << zbits;
+                zbits += R;
+                if (zbits >= 32) { wout[zk++] = (uint32_t)zacc; zacc >>= 32; zbits -= 32; }
             }
         }
+        (void)acc; (void)junk; (void)nbits; (void)kw;
+
+        // the stores of the previous tile must have read the staging buffer
+        if (tid == 0) bulk_wait_read0();
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<float4*>(hout_row + (((uint32_t)c << 4) ^ sw)) = H[c];
         if constexpr (R % 4 == 0) {
 #pragma unroll
             for (int q = 0; q < R / 4; ++q)
@@ -310,8 +365,9 @@ encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
         fence_proxy_async_smem();               // my writes -> visible to the TMA stores
         __syncthreads();
         if (tid == 0) {
-            tma_store_2d(&tm_h, 0, (int)(tile * kTileRows), base + L::kHoutOff);
-            bulk_store_1d(codes + (uint64_t)tile * (R * kTileRows), base + L::kCoutOff, L::kCodeBytes);
+            tma_store_2d(&bt.tm_h[entry], 0, (int)(tile * kTileRows), base + L::kHoutOff);
+            bulk_store_1d(bt.codes[entry] + (uint64_t)tile * (R * kTileRows), base + L::kCoutOff,
+                          L::kCodeBytes);
             bulk_commit();
         }
     }
@@ -322,14 +378,18 @@ encode_tiled_kernel(const __grid_constant__ CUtensorMap tm_g, const __grid_const
     __syncthreads();
     if (*s_abort) return;
 
-    // ragged end: the buckets after the last whole tile, spread over the CTAs from
-    // the back of the grid
+    // ragged ends: the buckets after the last whole tile of every vector, spread over the
+    // CTAs from the back of the grid
     const uint64_t tail_first = (uint64_t)n_tiles * buckets_per_tile;
     const uint64_t nb_total = (P.d + P.bucket - 1) / P.bucket;
+    const uint64_t n_tail = nb_total - tail_first;
     uint32_t* s_red = reinterpret_cast<uint32_t*>(sm);   // the buffers are idle now
-    for (uint64_t b = tail_first + (gridDim.x - 1 - blockIdx.x); b < nb_total; b += gridDim.x)
-        encode_bucket_generic<kEncodeThreads>(P, b, worker, step, g, h, codes, scales, status,
+    for (uint64_t k = gridDim.x - 1 - blockIdx.x; k < n_tail * n_workers; k += gridDim.x) {
+        const uint32_t e = (uint32_t)(k / n_tail);
+        encode_bucket_generic<kEncodeThreads>(P, tail_first + (k - e * n_tail), worker_base + e, step,
+                                              bt.g[e], bt.h[e], bt.codes[e], bt.scales[e], status,
                                               s_red, tid);
+    }
 }
 
 }  // namespace ecq

@@ -62,6 +62,11 @@ class GpuCodec:
         ecq.ecq_encode(self.ctx, worker, step, grad, self.err[worker][1],
                        self.codes[worker][1], self.scales[worker][1])
 
+    def encode_batch(self, step, grads):
+        W = len(grads)
+        ecq.ecq_encode_batch(self.ctx, step, grads, [e[1] for e in self.err[:W]],
+                             [c[1] for c in self.codes[:W]], [s[1] for s in self.scales[:W]])
+
     def decode(self, W=None):
         W = W or self.W
         ecq.ecq_decode_mean(self.ctx, [c[1] for c in self.codes[:W]],
@@ -79,7 +84,7 @@ def codes_np(t: torch.Tensor) -> np.ndarray:
 
 
 def full_parity(d, bucket, s, alpha, beta, seed, W, steps, grad_fn, mode=0, err0=None,
-                expect_status=ecq.ECQ_OK, check_decode=True):
+                expect_status=ecq.ECQ_OK, check_decode=True, batch=False):
     """Element-by-element comparison over whole vectors.
 
     ``grad_fn(worker, step)`` returns a float32 CUDA tensor of d entries.
@@ -93,8 +98,11 @@ def full_parity(d, bucket, s, alpha, beta, seed, W, steps, grad_fn, mode=0, err0
                 h_or[w] = err0[w].cpu().numpy().copy()
         for t in range(steps):
             grads = [grad_fn(w, t) for w in range(W)]
-            for w in range(W):
-                gpu.encode(w, t, grads[w])
+            if batch:
+                gpu.encode_batch(t, grads)
+            else:
+                for w in range(W):
+                    gpu.encode(w, t, grads[w])
             if check_decode:
                 gpu.decode()
             st = gpu.status()

@@ -42,12 +42,22 @@ def test_many_tiles_more_than_one_wave(bucket, s):
                 check_decode=True)
 
 
+@pytest.mark.parametrize("bucket,s,W", [(512, 4, 4), (4096, 8, 3), (128, 1, 8), (96, 2, 2), (1024, 128, 64)])
+def test_batched_encode_is_one_launch_with_the_same_result(bucket, s, W):
+    d = 4096 * 7 + 2 * bucket + 12
+    before = ecq.ecq_launch_count()
+    full_parity(d, bucket, s, 1.0, 0.9, SEED, W=W, steps=2, grad_fn=randn_fn(d, base=W), batch=True)
+    launches = ecq.ecq_launch_count() - before
+    tiled = (bucket & (bucket - 1)) == 0 and bucket <= 4096
+    assert launches == 2 * ((1 if tiled else W) + 1)
+
+
 def test_alpha_beta_variants_and_mode1():
     d = 4096 * 3 + 777
     for alpha, beta in ((0.0, 0.0), (0.2, 0.9), (0.01, 1.0), (1.0, 0.99), (2.5, 0.5)):
         for mode in (0, 1):
             full_parity(d, 512, 4, alpha, beta, 99, W=2, steps=4, grad_fn=randn_fn(d, base=3),
-                        mode=mode)
+                        mode=mode, batch=(mode == 1))
 
 
 def test_worker_step_seed_select_the_stream():
@@ -191,14 +201,14 @@ def _sampled_config(w, steps, W=None, ranges=None, grads=None):
     so = SampledOracle(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, W, ranges)
     try:
         for t in range(steps):
+            gs = [grads(p, t) if grads else wl.gradient(w, p, t, "cuda") for p in range(W)]
+            before = gpu.err[0][1].clone()
+            gpu.encode_batch(t, gs)                 # the launch configuration bench.py times
+            whole_vector_properties(gpu, 0, gs[0], before, w.alpha)
+            del before
             for p in range(W):
-                g = grads(p, t) if grads else wl.gradient(w, p, t, "cuda")
-                before = gpu.err[p][1].clone() if p == 0 else None
-                gpu.encode(p, t, g)
-                if p == 0:
-                    whole_vector_properties(gpu, p, g, before, w.alpha)
-                so.encode_and_compare(gpu, p, t, g)
-                del g
+                so.encode_and_compare(gpu, p, t, gs[p])
+            del gs
             gpu.decode(W)
             assert gpu.status() == ecq.ECQ_OK
             so.decode_and_compare(gpu)
