@@ -38,9 +38,11 @@ METRIC = "codec_step_throughput"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes per launch of the tiled encode kernel from an ncu capture, keyed by
-# workload; None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes per entry of the batched tiled encode kernel from an ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum over 817,825,024 entries; see
+# profiles/encode_tiled_kernel_resnet50.md), keyed by (bucket, levels).  Traffic grows in
+# proportion to the entries of a launch.  Set an entry to None when the kernel changes.
+NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): 10192464896 / 817825024}
 
 
 def code_bits(s: int) -> int:
@@ -340,7 +342,9 @@ def main():
             "roofline": {"kernel": "encode_tiled_kernel", "bound": "hbm", "achieved": enc_gbs,
                          "peak": peak, "peak_source": "of " + how, "unit": "GB/s",
                          "frac": enc_gbs / peak,
-                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, w.bucket, w.s))},
+                         "traffic": (NCU_DRAM_BYTES_PER_ENTRY[(w.bucket, w.s)] * W * d
+                                     if NCU_DRAM_BYTES_PER_ENTRY.get((w.bucket, w.s)) else None),
+                         "algorithmic_bytes_per_launch": W * enc_bytes},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
