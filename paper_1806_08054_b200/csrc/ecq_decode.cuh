@@ -153,7 +153,9 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
     constexpr uint32_t mask = (1u << R) - 1u;
     extern __shared__ __align__(128) uint8_t dsm[];
     const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
+    // broadcast from lane 0: the compiler then knows the value is warp-uniform and keeps the
+    // per-warp bookkeeping (ring slots, unit counters, pointers) on the uniform datapath
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
     uint8_t* const ring = dsm + warp * L::kWarpBytes;
     uint8_t* const stage = ring + D * L::kUnitBytes;
     float2* const a_tab = reinterpret_cast<float2*>(stage + 4096);
