@@ -60,18 +60,29 @@ struct ecq_ctx {
 
 namespace {
 
-// One row of the tiled view is 32 floats; a box is a whole tile of 128 rows.
+// One row of the tiled view is 32 floats; a box is a whole tile of 128 rows.  A map is a
+// pure function of (base, rows), and encoding one costs microseconds on the host, which
+// would dominate small vectors: each host thread keeps the maps it made in a small
+// direct-mapped cache.
 bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
+    struct Entry { const float* base; uint64_t rows; CUtensorMap map; };
+    constexpr unsigned kEntries = 256;
+    thread_local Entry cache[kEntries];          // zero-initialised: base == nullptr is empty
+    const uintptr_t a = reinterpret_cast<uintptr_t>(base);
+    Entry& e = cache[((a >> 8) ^ (a >> 16) ^ (a >> 24)) & (kEntries - 1)];
+    if (e.base == base && e.rows == rows) { *tm = e.map; return true; }
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {32, rows};
     const cuuint64_t strides[1] = {128};
     const cuuint32_t box[2] = {32, (cuuint32_t)kTileRows};
     const cuuint32_t estr[2] = {1, 1};
-    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides,
-               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-           CUDA_SUCCESS;
+    if (enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides,
+            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    e.base = base; e.rows = rows; e.map = *tm;
+    return true;
 }
 
 // Buffers of one batch entry as the launchers see them.
