@@ -141,6 +141,19 @@ int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
                     const float* const* scales, float* out, void* cuda_stream);
 
 /*
+ * Receiver side with the model update fused in (Algorithm 1, "compute global
+ * gradients" followed by "update model parameters w(t+1) = w(t) - eta * g~(t)"):
+ *   g~_i     = the mean ecq_decode_mean would produce
+ *   params_i <- fma(-eta, g~_i, params_i)       (one rounding)
+ *   out_i    = g~_i when out is not NULL
+ *   params [d]  in/out, 16-byte aligned; out [d] or NULL, must not alias params
+ * Saves the separate pass over the decoded gradient that an optimiser step would make.
+ */
+int ecq_decode_mean_update(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
+                           const float* const* scales, float eta, float* params, float* out,
+                           void* cuda_stream);
+
+/*
  * One whole iteration from HOST gradients to a HOST result: for every worker
  * copy its gradient to the device, ecq_encode it, then ecq_decode_mean all W
  * messages and copy the mean back.  Copies of worker w+1 overlap the encode of

@@ -64,6 +64,8 @@ def _load():
         lib.ecqo_encode_given_draws.restype = i32
         lib.ecqo_decode_mean.argtypes = [u64, u32, u32, u32, vp, vp, vp]
         lib.ecqo_decode_mean.restype = i32
+        lib.ecqo_decode_mean_update.argtypes = [u64, u32, u32, u32, vp, vp, f32, vp, vp]
+        lib.ecqo_decode_mean_update.restype = i32
         lib.ecqo_unpack_levels.argtypes = [u64, u32, vp, vp]
         lib.ecqo_unpack_levels.restype = None
         _lib = lib
@@ -145,6 +147,23 @@ def decode_mean(codes: Sequence[np.ndarray], scales: Sequence[np.ndarray], *,
     rc = _load().ecqo_decode_mean(n, bucket, s, W, cp, sp, _ptr(out))
     if rc != 0:
         raise ValueError("oracle decode_mean: bad arguments")
+    return out
+
+
+def decode_mean_update(codes: Sequence[np.ndarray], scales: Sequence[np.ndarray], params: np.ndarray,
+                       *, eta: float, bucket: int, s: int) -> np.ndarray:
+    """Eq. 4 then Algorithm 1's update: ``params`` is updated IN PLACE to
+    ``params - eta * mean`` (one fused multiply-add per entry); returns the mean."""
+    W, n = len(codes), params.size
+    assert params.dtype == np.float32 and params.flags.c_contiguous
+    cs = [np.ascontiguousarray(c, dtype=np.uint32) for c in codes]
+    ss = [np.ascontiguousarray(x, dtype=np.float32) for x in scales]
+    cp = (ctypes.c_void_p * W)(*[_ptr(c) for c in cs])
+    sp = (ctypes.c_void_p * W)(*[_ptr(x) for x in ss])
+    out = np.zeros(n, dtype=np.float32)
+    rc = _load().ecqo_decode_mean_update(n, bucket, s, W, cp, sp, eta, _ptr(params), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle decode_mean_update: bad arguments")
     return out
 
 

@@ -23,6 +23,8 @@
 // Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11), written
 // here from its published round function.
 //
+//   decode_mean_update  the same followed by Algorithm 1's "update model parameters".
+//
 // Parity pins (tests/test_oracle_*.py): Philox known answers; closed forms for
 // r and the message length; hand-worked level-boundary inputs; exact-rational
 // threshold checks of the rounding law; brute-force expectation on d = 8;
@@ -245,6 +247,21 @@ int ecqo_decode_mean(uint64_t n, uint32_t B, uint32_t s, uint32_t W,
             acc = std::fmaf((float)q, a, acc);
         }
         out[i] = acc / (float)W;
+    }
+    return 0;
+}
+
+// Algorithm 1, "update model parameters": w <- w - eta * g~, with g~ the mean above,
+// as one fused multiply-add per entry.
+int ecqo_decode_mean_update(uint64_t n, uint32_t B, uint32_t s, uint32_t W,
+                            const uint32_t* const* codes, const float* const* scales,
+                            float eta, float* params, float* out) {
+    std::vector<float> mean(n);
+    const int rc = ecqo_decode_mean(n, B, s, W, codes, scales, mean.data());
+    if (rc != 0) return rc;
+    for (uint64_t i = 0; i < n; ++i) {
+        params[i] = std::fmaf(-eta, mean[i], params[i]);
+        if (out) out[i] = mean[i];
     }
     return 0;
 }

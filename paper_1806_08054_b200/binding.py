@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.ecq_encode_batch.restype = i32
         L.ecq_decode_mean.argtypes = [vp, u32, vp, vp, vp, vp]
         L.ecq_decode_mean.restype = i32
+        L.ecq_decode_mean_update.argtypes = [vp, u32, vp, vp, f32, vp, vp, vp]
+        L.ecq_decode_mean_update.restype = i32
         L.ecq_step_host_workspace_bytes.argtypes = [vp, u32]
         L.ecq_step_host_workspace_bytes.restype = u64
         L.ecq_step_host.argtypes = [vp, u32, u32, vp, vp, vp, u64, vp, vp]
@@ -157,6 +159,19 @@ def ecq_decode_mean(ctx: int, codes: Sequence[torch.Tensor], scales: Sequence[to
     rc = lib().ecq_decode_mean(ctx, W, cp, sp, _dev(out, torch.float32, "out"), _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_decode_mean")
+
+
+def ecq_decode_mean_update(ctx: int, codes: Sequence[torch.Tensor], scales: Sequence[torch.Tensor],
+                           eta: float, params: torch.Tensor, out=None, stream=None) -> None:
+    """Receiver-side kernel with ``params <- params - eta * mean`` fused in."""
+    W = len(codes)
+    cp = (ctypes.c_void_p * W)(*[_dev(c, torch.int32, "codes") for c in codes])
+    sp = (ctypes.c_void_p * W)(*[_dev(s, torch.float32, "scales") for s in scales])
+    rc = lib().ecq_decode_mean_update(ctx, W, cp, sp, eta, _dev(params, torch.float32, "params"),
+                                      None if out is None else _dev(out, torch.float32, "out"),
+                                      _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_decode_mean_update")
 
 
 def ecq_step_host_workspace_bytes(ctx: int, W: int) -> int:

@@ -184,7 +184,7 @@ int encode_impl(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, floa
 }
 
 template <int R>
-void launch_decode(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, cudaStream_t st,
+void launch_decode(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out, cudaStream_t st,
                    float w_recip, int w_pow2) {
     constexpr int G = DecodeGroup<R>::kElems;
     const uint64_t n_groups = (c->P.d + G - 1) / G;
@@ -197,7 +197,7 @@ void launch_decode(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, 
 
 // Tiled decode: returns false when the shape is not covered (caller falls back).
 template <int R>
-bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out,
+bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out,
                          cudaStream_t st, float w_recip, int w_pow2) {
     using L = DecodeTiled<R>;
     const uint32_t B = c->P.bucket;
@@ -228,7 +228,7 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, float*
     return true;
 }
 
-int decode_impl(ecq_ctx* c, uint32_t W, const MessageTable& tab, float* out, cudaStream_t st) {
+int decode_impl(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out, cudaStream_t st) {
     const int w_pow2 = (W & (W - 1)) == 0;
     const float w_recip = 1.0f / (float)W;
     bool done = false;
@@ -370,7 +370,24 @@ int ecq_decode_mean(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,
         tab.codes[w] = codes[w];
         tab.scales[w] = scales[w];
     }
-    return decode_impl(c, W, tab, out, static_cast<cudaStream_t>(cuda_stream));
+    return decode_impl(c, W, tab, DecodeOut{out, nullptr, 0.f}, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ecq_decode_mean_update(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,
+                           const float* const* scales, float eta, float* params, float* out,
+                           void* cuda_stream) {
+    if (!c || !codes || !scales || !params || W == 0 || W > ECQ_MAX_WORKERS) return ECQ_ERR_ARG;
+    if (!aligned16(params) || (out && !aligned16(out)) || !(eta == eta) || params == out)
+        return ECQ_ERR_ARG;
+    MessageTable tab;
+    std::memset(&tab, 0, sizeof(tab));
+    for (uint32_t w = 0; w < W; ++w) {
+        if (!codes[w] || !scales[w] || !aligned16(codes[w]) || !aligned4(scales[w]))
+            return ECQ_ERR_ARG;
+        tab.codes[w] = codes[w];
+        tab.scales[w] = scales[w];
+    }
+    return decode_impl(c, W, tab, DecodeOut{out, params, -eta}, static_cast<cudaStream_t>(cuda_stream));
 }
 
 uint64_t ecq_step_host_workspace_bytes(const ecq_ctx* c, uint32_t W) {
@@ -433,7 +450,7 @@ int ecq_step_host(ecq_ctx* c, uint32_t W, uint32_t step, const float* const* gra
         rc = encode_impl(c, w, step, stage[sl], err_dev + (uint64_t)w * d, codes, scales, st);
         cudaEventRecord(c->ev_encoded[sl], st);
     }
-    if (rc == ECQ_OK) rc = decode_impl(c, W, tab, out_dev, st);
+    if (rc == ECQ_OK) rc = decode_impl(c, W, tab, DecodeOut{out_dev, nullptr, 0.f}, st);
     if (rc == ECQ_OK &&
         cudaMemcpyAsync(out_host, out_dev, d * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         rc = ECQ_ERR_CUDA;
@@ -559,7 +576,7 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
         tab.scales[w] = scales;
         rc = encode_impl(&c, w, step, grads[w], err + (uint64_t)w * d, codes, scales, st);
     }
-    if (rc == ECQ_OK) rc = decode_impl(&c, W, tab, out, st);
+    if (rc == ECQ_OK) rc = decode_impl(&c, W, tab, DecodeOut{out, nullptr, 0.f}, st);
     uint32_t bits = 0;
     if (cudaMemcpyAsync(&bits, c.d_status, sizeof(bits), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)

@@ -11,6 +11,27 @@ struct MessageTable {
     const float* scales[64];
 };
 
+// Where a decoded mean goes: to `out` (may be null), and, for the fused model update of
+// Algorithm 1 ("update model parameters w <- w - eta * g~"), into `params` (may be null).
+struct DecodeOut {
+    float* out;
+    float* params;
+    float neg_eta;
+};
+__device__ __forceinline__ void emit1(const DecodeOut& o, uint64_t i, float v) {
+    if (o.params) o.params[i] = __fmaf_rn(o.neg_eta, v, o.params[i]);
+    if (o.out) o.out[i] = v;
+}
+__device__ __forceinline__ void emit4(const DecodeOut& o, uint64_t i, float4 v) {
+    if (o.params) {
+        float4 p = *reinterpret_cast<const float4*>(o.params + i);
+        p.x = __fmaf_rn(o.neg_eta, v.x, p.x); p.y = __fmaf_rn(o.neg_eta, v.y, p.y);
+        p.z = __fmaf_rn(o.neg_eta, v.z, p.z); p.w = __fmaf_rn(o.neg_eta, v.w, p.w);
+        *reinterpret_cast<float4*>(o.params + i) = p;
+    }
+    if (o.out) *reinterpret_cast<float4*>(o.out + i) = v;
+}
+
 // Entries per thread: the shortest run whose codes fill whole 32-bit words.
 template <int R> struct DecodeGroup {
     static constexpr int kElems = (R % 8 == 0) ? 4 : (R % 4 == 0) ? 8 : (R % 2 == 0) ? 16 : 32;
@@ -22,7 +43,7 @@ template <int R> struct DecodeGroup {
 template <int R>
 __global__ void __launch_bounds__(256)
 decode_mean_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
-                   float* __restrict__ out, const uint64_t n_groups, const uint64_t n_words,
+                   const DecodeOut dst, const uint64_t n_groups, const uint64_t n_words,
                    const float w_recip, const int w_pow2) {
     constexpr int G = DecodeGroup<R>::kElems;
     constexpr int NW = DecodeGroup<R>::kWords;
@@ -59,12 +80,11 @@ decode_mean_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         if (i0 + G <= P.d) {
 #pragma unroll
             for (int j = 0; j < G; j += 4)
-                *reinterpret_cast<float4*>(out + i0 + j) =
-                    make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                emit4(dst, i0 + j, make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]));
         } else {
 #pragma unroll
             for (int j = 0; j < G; ++j)
-                if (i0 + j < P.d) out[i0 + j] = acc[j];
+                if (i0 + j < P.d) emit1(dst, i0 + j, acc[j]);
         }
     }
 }
@@ -72,7 +92,7 @@ decode_mean_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
 // Any code width (r up to 16): 32 entries per thread, run-time shifts.
 __global__ void __launch_bounds__(256)
 decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
-                           const __grid_constant__ MessageTable tab, float* __restrict__ out,
+                           const __grid_constant__ MessageTable tab, const DecodeOut dst,
                            const uint64_t n_groups, const uint64_t n_words, const float w_recip,
                            const int w_pow2) {
     const uint32_t r = P.r, mask = (1u << r) - 1u;
@@ -94,7 +114,7 @@ decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
                 const float q = __fsub_rn(__uint_as_float(0x4B000000u | c), magic);
                 acc = __fmaf_rn(q, a, acc);
             }
-            out[i0 + j] = w_pow2 ? __fmul_rn(acc, w_recip) : __fdiv_rn(acc, (float)W);
+            emit1(dst, i0 + j, w_pow2 ? __fmul_rn(acc, w_recip) : __fdiv_rn(acc, (float)W));
         }
     }
 }
@@ -145,7 +165,7 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
 template <int R>
 __global__ void __launch_bounds__(kDecWarps * 32)
 decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
-                    float* __restrict__ out, const uint32_t n_tiles, const uint64_t n_words,
+                    const DecodeOut dst, const uint32_t n_tiles, const uint64_t n_words,
                     const float w_recip, const int w_pow2, const uint32_t exp23_bits) {
     using L = DecodeTiled<R>;
     constexpr int D = L::kRing;
@@ -307,12 +327,12 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
             *reinterpret_cast<float4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) =
                 make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
         __syncwarp();
-        float* o = out + (uint64_t)tile * kDecTileElems;
+        const uint64_t o = (uint64_t)tile * kDecTileElems;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
             const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
-            *reinterpret_cast<float4*>(o + idx * 4) = v;
+            emit4(dst, o + idx * 4, v);
         }
         __syncwarp();
     }
@@ -333,7 +353,7 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
             const uint32_t c = __funnelshift_r(lo, hi1, sh) & mask;
             acc1 = __fmaf_rn(__fsub_rn(__uint_as_float(0x4B000000u | c), magic), a, acc1);
         }
-        out[i] = w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, (float)W);
+        emit1(dst, i, w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, (float)W));
     }
 }
 

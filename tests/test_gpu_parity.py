@@ -123,6 +123,42 @@ def test_decode_worker_counts():
         full_parity(d, B, s, 1.0, 0.9, SEED, W=W, steps=1, grad_fn=randn_fn(d, base=W))
 
 
+@pytest.mark.parametrize("bucket,s,W,d", [(512, 4, 4, 4096 * 5 + 700), (2048, 1, 16, 4096 * 3 + 2048 + 24),
+                                            (96, 8, 3, 5000), (128, 300, 2, 3000), (512, 8, 8, 777)])
+def test_fused_model_update(bucket, s, W, d):
+    # Algorithm 1, last line, fused into the receiver kernel: bit-exact against the oracle
+    # (same operations in the same order), with and without the mean being written out
+    gpu = GpuCodec(d, bucket, s, 1.0, 0.9, SEED, W)
+    fn = randn_fn(d, base=d + W)
+    grads = [fn(w, 0) for w in range(W)]
+    gpu.encode_batch(0, grads)
+    msgs = []
+    for w in range(W):
+        h = np.zeros(d, np.float32)
+        c, sc, _ = oracle.encode(grads[w].cpu().numpy(), h, bucket=bucket, s=s, alpha=1.0, beta=0.9,
+                                 seed=SEED, worker=w, step=0)
+        msgs.append((c, sc))
+    gen = torch.Generator(device="cuda"); gen.manual_seed(3)
+    p0 = torch.randn(d, generator=gen, device="cuda")
+    for eta, with_out in ((0.02, True), (1.0, False), (0.0, True)):
+        params = p0.clone()
+        if with_out:
+            gpu.out[1].fill_(-7.0)
+        ecq.ecq_decode_mean_update(gpu.ctx, [c[1] for c in gpu.codes], [x[1] for x in gpu.scales], eta,
+                                   params, gpu.out[1] if with_out else None)
+        assert gpu.status() == ecq.ECQ_OK
+        p_or = p0.cpu().numpy().copy()
+        mean = oracle.decode_mean_update([m[0] for m in msgs], [m[1] for m in msgs], p_or, eta=eta,
+                                         bucket=bucket, s=s)
+        assert np.array_equal(params.cpu().numpy().view(np.uint32), p_or.view(np.uint32))
+        if with_out:
+            assert close(gpu.out[1].cpu().numpy(), mean)
+    gpu.check_guards()
+    L = ecq.binding.lib()
+    assert L.ecq_decode_mean_update(gpu.ctx, W, None, None, 0.1, None, None, None) == ecq.ECQ_ERR_ARG
+    gpu.close()
+
+
 def test_argument_errors():
     with pytest.raises(ecq.EcqError):
         ecq.ecq_create(0, 512, 4, 1.0, 0.9, 1)

@@ -387,3 +387,39 @@ def test_decode_exact_integer_case_and_fp64():
     # fp32 partial sums carry rounding errors relative to the largest scale
     top = max(float(x.max()) for x in scl)
     assert np.allclose(out, acc / W, rtol=1e-6, atol=2.0 ** -22 * top)
+
+
+# ------------------------------------------------- fused model update --------
+def test_decode_mean_update_is_algorithm1_last_line():
+    # w <- w - eta * mean: eta = 0 leaves w alone; power-of-two data makes every operation
+    # exact (compare with integers); otherwise compare with an independent fp64 evaluation
+    rng = np.random.default_rng(31)
+    n, B, s, W = 512, 64, 4, 4
+    msgs, scl, ints = [], [], []
+    for w in range(W):
+        g = rng.integers(-s, s + 1, n).astype(np.float32)
+        g[::B] = s                                     # scale = s exactly -> level step 1
+        c, sc, _ = enc(g, np.zeros(n, np.float32), bucket=B, s=s, worker=w)
+        msgs.append(c); scl.append(sc); ints.append(g.astype(np.int64))
+    mean = oracle.decode_mean(msgs, scl, n=n, bucket=B, s=s)
+    p0 = rng.integers(-100, 100, n).astype(np.float32)
+    p = p0.copy()
+    out = oracle.decode_mean_update(msgs, scl, p, eta=0.0, bucket=B, s=s)
+    assert np.array_equal(p, p0) and np.array_equal(out, mean)
+    p = p0.copy()
+    oracle.decode_mean_update(msgs, scl, p, eta=0.5, bucket=B, s=s)
+    assert np.array_equal(p * 8, p0 * 8 - sum(ints).astype(np.float32))     # 0.5 * (sum / 4) exact
+    # generic values: one rounding away from the exact w - eta * mean
+    msgs, scl = [], []
+    for w in range(W):
+        g = (rng.standard_normal(n) * 0.05).astype(np.float32)
+        c, sc, _ = enc(g, np.zeros(n, np.float32), bucket=B, s=s, worker=w)
+        msgs.append(c); scl.append(sc)
+    mean = oracle.decode_mean(msgs, scl, n=n, bucket=B, s=s).astype(np.float64)
+    p0 = rng.standard_normal(n).astype(np.float32)
+    p = p0.copy()
+    eta = np.float32(0.02)
+    oracle.decode_mean_update(msgs, scl, p, eta=float(eta), bucket=B, s=s)
+    exact = p0.astype(np.float64) - float(eta) * mean
+    assert np.all(np.abs(p - exact) <= 0.5 * np.spacing(np.abs(exact).astype(np.float32)) * 1.0001)
+    assert not np.array_equal(p, p0)
