@@ -282,6 +282,10 @@ def main():
     total_ms = ev[0].elapsed_time(ev[-1])
     enc_ms = sum(ev[t].elapsed_time(mids[t]) for t in range(args.steps))
     dec_ms = sum(mids[t].elapsed_time(ev[t + 1]) for t in range(args.steps))
+    # level statistics of worker 0's last message (outside the timed region)
+    counts = torch.zeros(2 * w.s + 1, dtype=torch.int64, device="cuda")
+    ecq.ecq_code_histogram(ctx, codes[0], counts)
+    entropy_bits = ecq.ecq_entropy_bound_bits(counts.cpu().tolist())
     status = ecq.ecq_status(ctx)
     if status != ecq.ECQ_OK:
         raise SystemExit("codec status %d: %s" % (status, ecq.binding.strerror(status)))
@@ -348,6 +352,12 @@ def main():
                          "traffic": (NCU_DRAM_BYTES_PER_ENTRY[(w.bucket, w.s)] * W * d
                                      if NCU_DRAM_BYTES_PER_ENTRY.get((w.bucket, w.s)) else None),
                          "algorithmic_bytes_per_launch": W * enc_bytes},
+            "message": {"fixed_bits_per_entry": r + 32.0 / w.bucket,
+                        "compression_fixed": 32.0 / (r + 32.0 / w.bucket),
+                        "entropy_bound_bits_per_entry": (entropy_bits + 32.0 * nb) / d,
+                        "compression_entropy_bound": 32.0 * d / (entropy_bits + 32.0 * nb),
+                        "note": "worker 0, last timed step; the paper's Table 1 ratios are "
+                                "entropy-coded on other workloads (context only)"},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }

@@ -154,6 +154,18 @@ int ecq_decode_mean_update(ecq_ctx* ctx, uint32_t W, const uint32_t* const* code
                            void* cuda_stream);
 
 /*
+ * Level statistics of one message (paragraph after Eq. 9: with d_k entries on the k-th
+ * of the 2s+1 levels, an entropy code needs at most sum_k d_k log2(d / d_k) bits).
+ *   codes   [ecq_codes_words()] device, one worker's code stream
+ *   counts  [2s+1] device uint64, 8-byte aligned: counts[k] = entries whose level is k - s;
+ *           zeroed and filled by the call (asynchronously on the stream)
+ */
+int ecq_code_histogram(ecq_ctx* ctx, const uint32_t* codes, uint64_t* counts, void* cuda_stream);
+
+/* sum_k d_k log2(d / d_k) over the non-empty bins of HOST counts, d = sum_k d_k. */
+double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins);
+
+/*
  * One whole iteration from HOST gradients to a HOST result: for every worker
  * copy its gradient to the device, ecq_encode it, then ecq_decode_mean all W
  * messages and copy the mean back.  Copies of worker w+1 overlap the encode of

@@ -66,6 +66,10 @@ def _load():
         lib.ecqo_decode_mean.restype = i32
         lib.ecqo_decode_mean_update.argtypes = [u64, u32, u32, u32, vp, vp, f32, vp, vp]
         lib.ecqo_decode_mean_update.restype = i32
+        lib.ecqo_code_histogram.argtypes = [u64, u32, vp, vp]
+        lib.ecqo_code_histogram.restype = None
+        lib.ecqo_entropy_bound_bits.argtypes = [vp, u32]
+        lib.ecqo_entropy_bound_bits.restype = ctypes.c_double
         lib.ecqo_unpack_levels.argtypes = [u64, u32, vp, vp]
         lib.ecqo_unpack_levels.restype = None
         _lib = lib
@@ -165,6 +169,20 @@ def decode_mean_update(codes: Sequence[np.ndarray], scales: Sequence[np.ndarray]
     if rc != 0:
         raise ValueError("oracle decode_mean_update: bad arguments")
     return out
+
+
+def code_histogram(codes: np.ndarray, *, n: int, s: int) -> np.ndarray:
+    """d_k, k < 2s+1: entries of the message on level k - s."""
+    c = np.ascontiguousarray(codes, dtype=np.uint32)
+    counts = np.zeros(2 * s + 1, dtype=np.uint64)
+    _load().ecqo_code_histogram(n, s, _ptr(c), _ptr(counts))
+    return counts
+
+
+def entropy_bound_bits(counts: np.ndarray) -> float:
+    """sum_k d_k log2(d / d_k) (paragraph after Eq. 9)."""
+    c = np.ascontiguousarray(counts, dtype=np.uint64)
+    return float(_load().ecqo_entropy_bound_bits(_ptr(c), c.size))
 
 
 def unpack_levels(codes: np.ndarray, *, n: int, s: int) -> np.ndarray:

@@ -266,6 +266,25 @@ int ecqo_decode_mean_update(uint64_t n, uint32_t B, uint32_t s, uint32_t W,
     return 0;
 }
 
+// Level counts d_k of one message and the entropy-coding bound of the paragraph after
+// Eq. 9: at most sum_k d_k log2(d / d_k) bits.
+void ecqo_code_histogram(uint64_t n, uint32_t s, const uint32_t* codes, uint64_t* counts) {
+    const uint32_t r = code_bits(s);
+    for (uint32_t k = 0; k < 2 * s + 1; ++k) counts[k] = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const uint32_t c = get_code(codes, i * r, r);
+        if (c < 2 * s + 1) counts[c] += 1;
+    }
+}
+
+double ecqo_entropy_bound_bits(const uint64_t* counts, uint32_t n_bins) {
+    double d = 0.0, bits = 0.0;
+    for (uint32_t k = 0; k < n_bins; ++k) d += (double)counts[k];
+    for (uint32_t k = 0; k < n_bins; ++k)
+        if (counts[k]) bits += (double)counts[k] * std::log2(d / (double)counts[k]);
+    return bits;
+}
+
 // Unpack one message into signed levels q_i (test helper for round trips).
 void ecqo_unpack_levels(uint64_t n, uint32_t s, const uint32_t* codes, int32_t* q) {
     const uint32_t r = code_bits(s);

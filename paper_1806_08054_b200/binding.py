@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.ecq_decode_mean.restype = i32
         L.ecq_decode_mean_update.argtypes = [vp, u32, vp, vp, f32, vp, vp, vp]
         L.ecq_decode_mean_update.restype = i32
+        L.ecq_code_histogram.argtypes = [vp, vp, vp, vp]
+        L.ecq_code_histogram.restype = i32
+        L.ecq_entropy_bound_bits.argtypes = [vp, u32]
+        L.ecq_entropy_bound_bits.restype = ctypes.c_double
         L.ecq_step_host_workspace_bytes.argtypes = [vp, u32]
         L.ecq_step_host_workspace_bytes.restype = u64
         L.ecq_step_host.argtypes = [vp, u32, u32, vp, vp, vp, u64, vp, vp]
@@ -172,6 +176,21 @@ def ecq_decode_mean_update(ctx: int, codes: Sequence[torch.Tensor], scales: Sequ
                                       _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_decode_mean_update")
+
+
+def ecq_code_histogram(ctx: int, codes: torch.Tensor, counts: torch.Tensor, stream=None) -> None:
+    """Fill ``counts`` (int64 CUDA tensor of 2s+1 entries) with the level counts of one message."""
+    rc = lib().ecq_code_histogram(ctx, _dev(codes, torch.int32, "codes"),
+                                  _dev(counts, torch.int64, "counts"), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_code_histogram")
+
+
+def ecq_entropy_bound_bits(counts_host) -> float:
+    """sum_k d_k log2(d / d_k) from host counts (any integer sequence)."""
+    n = len(counts_host)
+    arr = (ctypes.c_uint64 * n)(*[int(x) for x in counts_host])
+    return float(lib().ecq_entropy_bound_bits(arr, n))
 
 
 def ecq_step_host_workspace_bytes(ctx: int, W: int) -> int:

@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cstdint>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -13,6 +14,7 @@
 #include "ecq_common.cuh"
 #include "ecq_decode.cuh"
 #include "ecq_encode.cuh"
+#include "ecq_stats.cuh"
 
 using namespace ecq;
 
@@ -388,6 +390,36 @@ int ecq_decode_mean_update(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,
         tab.scales[w] = scales[w];
     }
     return decode_impl(c, W, tab, DecodeOut{out, params, -eta}, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int ecq_code_histogram(ecq_ctx* c, const uint32_t* codes, uint64_t* counts, void* cuda_stream) {
+    if (!c || !codes || !counts || !aligned16(codes) ||
+        (reinterpret_cast<uintptr_t>(counts) & 7u))
+        return ECQ_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const uint32_t nbins = 2 * c->P.s + 1;
+    if (cudaMemsetAsync(counts, 0, sizeof(uint64_t) * nbins, st) != cudaSuccess) return ECQ_ERR_CUDA;
+    const size_t smem = nbins <= kHistLaneBins ? (size_t)(kHistThreads / 32) * nbins * 32 * 4
+                      : nbins <= kHistSharedBins ? (size_t)nbins * 4 : 0;
+    const uint64_t rows = (c->P.d + 31) / 32;
+    uint64_t blocks = (rows + kHistThreads - 1) / kHistThreads;
+    const uint64_t cap = (uint64_t)c->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    code_histogram_kernel<<<(uint32_t)blocks, kHistThreads, smem, st>>>(
+        c->P, codes, reinterpret_cast<unsigned long long*>(counts));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins) {
+    if (!counts_host) return 0.0;
+    long double total = 0.0L;
+    for (uint32_t k = 0; k < n_bins; ++k) total += (long double)counts_host[k];
+    double bits = 0.0;
+    for (uint32_t k = 0; k < n_bins; ++k)
+        if (counts_host[k])
+            bits += (double)counts_host[k] * std::log2((double)total / (double)counts_host[k]);
+    return bits;
 }
 
 uint64_t ecq_step_host_workspace_bytes(const ecq_ctx* c, uint32_t W) {

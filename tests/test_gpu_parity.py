@@ -159,6 +159,24 @@ def test_fused_model_update(bucket, s, W, d):
     gpu.close()
 
 
+@pytest.mark.parametrize("bucket,s,d", [(512, 1, 4096 * 9 + 77), (512, 4, 4096 * 9 + 512 + 40), (96, 8, 5003),
+                                        (1024, 16, 33000), (4096, 128, 4096 * 6 + 1), (128, 300, 9000),
+                                        (32, 32767, 4099)])
+def test_code_histogram_and_entropy(bucket, s, d):
+    gpu = GpuCodec(d, bucket, s, 1.0, 0.9, SEED, 1)
+    gpu.encode(0, 0, randn_fn(d, base=s)(0, 0))
+    counts = torch.full((2 * s + 1,), -1, dtype=torch.int64, device="cuda")
+    ecq.ecq_code_histogram(gpu.ctx, gpu.codes[0][1], counts)
+    assert gpu.status() == ecq.ECQ_OK
+    ref = oracle.code_histogram(codes_np(gpu.codes[0][1]), n=d, s=s)
+    got = counts.cpu().numpy()
+    assert got.sum() == d and np.array_equal(got.astype(np.uint64), ref)
+    bits = ecq.ecq_entropy_bound_bits(got)
+    assert abs(bits - oracle.entropy_bound_bits(ref)) <= 1e-9 * max(bits, 1.0)
+    assert bits <= d * gpu.r + 1e-6
+    gpu.close()
+
+
 def test_argument_errors():
     with pytest.raises(ecq.EcqError):
         ecq.ecq_create(0, 512, 4, 1.0, 0.9, 1)

@@ -423,3 +423,22 @@ def test_decode_mean_update_is_algorithm1_last_line():
     exact = p0.astype(np.float64) - float(eta) * mean
     assert np.all(np.abs(p - exact) <= 0.5 * np.spacing(np.abs(exact).astype(np.float32)) * 1.0001)
     assert not np.array_equal(p, p0)
+
+
+# ------------------------------------------------- level statistics ----------
+def test_code_histogram_and_entropy_bound():
+    rng = np.random.default_rng(41)
+    for s, B, n in ((1, 128, 1000), (4, 512, 5000), (8, 96, 4001), (128, 4096, 9000)):
+        g = (rng.standard_normal(n) * 0.01).astype(np.float32)
+        codes, _, _ = enc(g, np.zeros(n, np.float32), bucket=B, s=s)
+        counts = oracle.code_histogram(codes, n=n, s=s)
+        ref = np.bincount(np_unpack(codes, n, oracle.code_bits(s)), minlength=2 * s + 1)
+        assert counts.sum() == n and np.array_equal(counts.astype(np.int64), ref)   # library bincount
+        d = counts.astype(np.float64)
+        nz = d > 0
+        assert abs(oracle.entropy_bound_bits(counts) - (d[nz] * np.log2(n / d[nz])).sum()) < 1e-6 * n
+    # closed forms: 2^k equally likely levels cost k bits per entry; one level costs nothing;
+    # and the bound never exceeds the fixed-width cost d * r
+    assert oracle.entropy_bound_bits(np.array([256] * 8, np.uint64)) == 8 * 256 * 3.0
+    assert oracle.entropy_bound_bits(np.array([0, 12345, 0], np.uint64)) == 0.0
+    assert oracle.entropy_bound_bits(np.array([10, 980, 10], np.uint64)) < 1000 * 2
