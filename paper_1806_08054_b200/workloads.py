@@ -191,3 +191,26 @@ def gradient(w: Workload, worker: int, step: int, device="cpu") -> torch.Tensor:
 
 def clear_cache() -> None:
     _lsq_cache.clear()
+
+
+class SynLinReg:
+    """Synthetic linear regression in the style of the paper's Syn-256/512/1024 runs
+    (Section 6.1): N samples x ~ N(0, I_d), y = <w*, x> + noise, split evenly over W workers.
+    The paper does not state the noise level; 0.1 is used here.  Only data and mini-batch
+    sampling live here; the optimiser loop belongs to whoever uses it."""
+
+    def __init__(self, d: int, W: int, seed: int, n_samples: int = 10_000, noise: float = 0.1,
+                 device="cuda"):
+        self.d, self.W = d, W
+        self.gen = _gen(770_000 + seed, torch.device(device))
+        self.X = torch.randn(n_samples, d, generator=self.gen, device=device)
+        self.w_star = torch.randn(d, generator=self.gen, device=device)
+        self.y = self.X @ self.w_star + noise * torch.randn(n_samples, generator=self.gen, device=device)
+        self.shards = torch.chunk(torch.arange(n_samples, device=device), W)
+
+    def minibatch_gradient(self, worker: int, w: torch.Tensor, batch: int = 64) -> torch.Tensor:
+        """Gradient of the mean squared error over a random mini-batch of the worker's shard."""
+        shard = self.shards[worker]
+        idx = shard[torch.randint(0, len(shard), (batch,), generator=self.gen, device=w.device)]
+        xb = self.X[idx]
+        return (xb.T @ (xb @ w - self.y[idx]) / batch).contiguous()
