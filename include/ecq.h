@@ -80,6 +80,21 @@ void ecq_destroy(ecq_ctx* ctx);
  */
 int ecq_set_error_mode(ecq_ctx* ctx, int mode);
 
+/*
+ * Choose the scaling factor ||v|| of Eq. 8 ("possible choices include l2-norm and
+ * l-infinity-norm"), taken per bucket.
+ *   0 (default)  l-infinity: max |v_i|
+ *   1            l2: sqrt(sum v_i^2).  The fp32 sum has a fixed order so that results do not
+ *                depend on the kernel's shape: every run of 32 consecutive entries is summed
+ *                front to back with one fused multiply-add per entry, the run sums are added
+ *                pairwise in index order, level by level.  Entries below about 1e-19 in
+ *                magnitude square to zero; a sum that overflows (entries beyond about 1e19)
+ *                is reported as ECQ_ERR_NONFINITE.  Buckets that are not a power of two
+ *                or exceed 4096 entries may have at most 32768 entries (else ECQ_ERR_ARG).
+ * The receiver side is the same for both.
+ */
+int ecq_set_norm(ecq_ctx* ctx, int norm);
+
 /* r = ceil(log2(2s+1)): bits per entry (paragraph after Eq. 9). */
 uint32_t ecq_code_bits(const ecq_ctx* ctx);
 /* nb = ceil(d / bucket): floats in one worker's `scales`. */

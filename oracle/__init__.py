@@ -56,10 +56,10 @@ def _load():
         lib.ecqo_num_buckets.restype = u64
         lib.ecqo_codes_words.argtypes = [u64, u32]
         lib.ecqo_codes_words.restype = u64
-        lib.ecqo_encode.argtypes = [u64, u32, u32, f32, f32, u64, i32, u32, u32, u64,
+        lib.ecqo_encode.argtypes = [u64, u32, u32, f32, f32, u64, i32, i32, u32, u32, u64,
                                     vp, vp, vp, vp, vp]
         lib.ecqo_encode.restype = i32
-        lib.ecqo_encode_given_draws.argtypes = [u64, u32, u32, f32, f32, i32,
+        lib.ecqo_encode_given_draws.argtypes = [u64, u32, u32, f32, f32, i32, i32,
                                                 vp, vp, vp, vp, vp, vp]
         lib.ecqo_encode_given_draws.restype = i32
         lib.ecqo_decode_mean.argtypes = [u64, u32, u32, u32, vp, vp, vp]
@@ -110,9 +110,10 @@ def codes_words(d: int, s: int) -> int:
 
 def encode(g: np.ndarray, h: np.ndarray, *, bucket: int, s: int, alpha: float,
            beta: float, seed: int, worker: int, step: int, mode: int = 0,
-           first_index: int = 0, draws: Optional[np.ndarray] = None):
+           first_index: int = 0, draws: Optional[np.ndarray] = None, norm: int = 0):
     """Encode one worker's slice; ``h`` is updated IN PLACE (Eq. 6).
 
+    ``norm`` 0 takes the l-infinity norm of the bucket as the scale of Eq. 8, 1 the l2 norm.
     Returns ``(codes uint32[words], scales float32[nb], status)``.  ``draws``
     (one uint32 per element) replaces the Philox stream when given.
     """
@@ -124,13 +125,13 @@ def encode(g: np.ndarray, h: np.ndarray, *, bucket: int, s: int, alpha: float,
     status = np.zeros(1, dtype=np.uint32)
     lib = _load()
     if draws is None:
-        rc = lib.ecqo_encode(n, bucket, s, alpha, beta, seed, mode, worker, step,
+        rc = lib.ecqo_encode(n, bucket, s, alpha, beta, seed, mode, norm, worker, step,
                              first_index, _ptr(g), _ptr(h), _ptr(codes), _ptr(scales),
                              _ptr(status))
     else:
         dr = np.ascontiguousarray(draws, dtype=np.uint32)
         assert dr.size == n
-        rc = lib.ecqo_encode_given_draws(n, bucket, s, alpha, beta, mode, _ptr(dr),
+        rc = lib.ecqo_encode_given_draws(n, bucket, s, alpha, beta, mode, norm, _ptr(dr),
                                          _ptr(g), _ptr(h), _ptr(codes), _ptr(scales),
                                          _ptr(status))
     if rc != 0:

@@ -9,7 +9,7 @@
 // What it computes, per worker p and iteration t, on a flat fp32 vector that is
 // cut into contiguous buckets of B entries (the last one may be shorter):
 //
-//   encode       Section 4: Eq. 7 (compensation), Eq. 8 with the l-infinity
+//   encode       Section 4: Eq. 7 (compensation), Eq. 8 with the l-infinity (or l2)
 //                scale taken per bucket, Eq. 9 (two-point stochastic rounding),
 //                Eq. 6 (incremental error accumulator), and the fixed-width
 //                r = ceil(log2(2s+1)) bit code of the paragraph after Eq. 9.
@@ -110,7 +110,7 @@ enum { STATUS_NONFINITE = 1u };
 // a large vector; `random_words`, when not null, replaces the Philox draw
 // (one word per element) so that tests can choose the draws.
 int encode_core(uint64_t n, uint32_t B, uint32_t s, float alpha, float beta,
-                uint64_t seed, int mode, uint32_t worker, uint32_t step,
+                uint64_t seed, int mode, int norm, uint32_t worker, uint32_t step,
                 uint64_t first_index, const uint32_t* random_words,
                 const float* g, float* h, uint32_t* codes, float* scales,
                 uint32_t* status) {
@@ -136,7 +136,27 @@ int encode_core(uint64_t n, uint32_t B, uint32_t s, float alpha, float beta,
             const uint32_t a = f2u(v[i - lo]) & 0x7FFFFFFFu;
             if (a > sbits) sbits = a;
         }
-        const float scale = u2f(sbits);
+        float scale = u2f(sbits);
+        if (norm == 1) {
+            // Eq. 8 with the l2 norm.  The fp32 sum of squares needs a stated order:
+            // each run of 32 consecutive entries is summed front to back with one fused
+            // multiply-add per entry, and the run sums are combined pairwise in index
+            // order, level by level (an odd one out is carried up unchanged).
+            std::vector<float> runs;
+            for (uint64_t i = lo; i < hi; i += 32) {
+                float acc = 0.0f;
+                for (uint64_t j = i; j < hi && j < i + 32; ++j) acc = std::fmaf(v[j - lo], v[j - lo], acc);
+                runs.push_back(acc);
+            }
+            while (runs.size() > 1) {
+                std::vector<float> up;
+                for (size_t k = 0; k < runs.size(); k += 2)
+                    up.push_back(k + 1 < runs.size() ? runs[k] + runs[k + 1] : runs[k]);
+                runs.swap(up);
+            }
+            sbits = f2u(runs[0]) & 0x7FFFFFFFu;       // NaN/Inf (also an overflowed sum) sort on top
+            scale = std::sqrt(runs[0]);
+        }
 
         bool zero_bucket = false;
         float inv = 0.0f, a_step = 0.0f;
@@ -216,17 +236,17 @@ uint64_t ecqo_num_buckets(uint64_t d, uint32_t B) { return (d + B - 1) / B; }
 uint64_t ecqo_codes_words(uint64_t d, uint32_t s) { return (d * code_bits(s) + 31) / 32; }
 
 int ecqo_encode(uint64_t n, uint32_t B, uint32_t s, float alpha, float beta,
-                uint64_t seed, int mode, uint32_t worker, uint32_t step,
+                uint64_t seed, int mode, int norm, uint32_t worker, uint32_t step,
                 uint64_t first_index, const float* g, float* h,
                 uint32_t* codes, float* scales, uint32_t* status) {
-    return encode_core(n, B, s, alpha, beta, seed, mode, worker, step, first_index,
+    return encode_core(n, B, s, alpha, beta, seed, mode, norm, worker, step, first_index,
                        nullptr, g, h, codes, scales, status);
 }
 
 int ecqo_encode_given_draws(uint64_t n, uint32_t B, uint32_t s, float alpha, float beta,
-                            int mode, const uint32_t* random_words, const float* g,
+                            int mode, int norm, const uint32_t* random_words, const float* g,
                             float* h, uint32_t* codes, float* scales, uint32_t* status) {
-    return encode_core(n, B, s, alpha, beta, 0, mode, 0, 0, 0, random_words, g, h,
+    return encode_core(n, B, s, alpha, beta, 0, mode, norm, 0, 0, 0, random_words, g, h,
                        codes, scales, status);
 }
 

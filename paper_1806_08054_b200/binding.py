@@ -46,6 +46,8 @@ def lib() -> ctypes.CDLL:
         L.ecq_destroy.restype = None
         L.ecq_set_error_mode.argtypes = [vp, i32]
         L.ecq_set_error_mode.restype = i32
+        L.ecq_set_norm.argtypes = [vp, i32]
+        L.ecq_set_norm.restype = i32
         L.ecq_code_bits.argtypes = [vp]
         L.ecq_code_bits.restype = u32
         L.ecq_num_buckets.argtypes = [vp]
@@ -115,6 +117,13 @@ def ecq_set_error_mode(ctx: int, mode: int) -> None:
     rc = lib().ecq_set_error_mode(ctx, mode)
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_set_error_mode")
+
+
+def ecq_set_norm(ctx: int, norm: int) -> None:
+    """0: l-infinity scale per bucket (default); 1: l2 scale (Eq. 8 allows either)."""
+    rc = lib().ecq_set_norm(ctx, norm)
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_set_norm")
 
 
 def ecq_code_bits(ctx: int) -> int:

@@ -284,7 +284,7 @@ int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels, floa
     ecq_ctx* c = new (std::nothrow) ecq_ctx();
     if (!c) return ECQ_ERR_ALLOC;
     CodecParams& P = c->P;
-    P.d = d; P.bucket = bucket; P.s = levels; P.mode = 0;
+    P.d = d; P.bucket = bucket; P.s = levels; P.mode = 0; P.norm = 0;
     P.alpha = alpha; P.beta = beta; P.sf = (float)levels;
     P.r = 0;
     while ((1ull << P.r) < 2ull * levels + 1ull) ++P.r;
@@ -329,6 +329,14 @@ void ecq_destroy(ecq_ctx* c) {
 int ecq_set_error_mode(ecq_ctx* c, int mode) {
     if (!c || (mode != 0 && mode != 1)) return ECQ_ERR_ARG;
     c->P.mode = mode;
+    return ECQ_OK;
+}
+
+int ecq_set_norm(ecq_ctx* c, int norm) {
+    if (!c || (norm != 0 && norm != 1)) return ECQ_ERR_ARG;
+    // the any-shape path sums at most kMaxL2Runs runs of 32 entries per bucket
+    if (norm == 1 && !c->tiled_ok && c->P.bucket > 32u * kMaxL2Runs) return ECQ_ERR_ARG;
+    c->P.norm = norm;
     return ECQ_OK;
 }
 
@@ -567,7 +575,7 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
     // a context on the stack: constants only, nothing allocated
     ecq_ctx c;
     CodecParams& P = c.P;
-    P.d = d; P.bucket = bucket; P.s = levels; P.mode = 0;
+    P.d = d; P.bucket = bucket; P.s = levels; P.mode = 0; P.norm = 0;
     P.alpha = alpha; P.beta = beta; P.sf = (float)levels;
     P.r = 0;
     while ((1ull << P.r) < 2ull * levels + 1ull) ++P.r;

@@ -16,6 +16,7 @@ struct CodecParams {
     uint32_t s;          // non-zero levels of Eq. 9
     uint32_t r;          // ceil(log2(2s+1))
     int32_t mode;        // 0: Eq. 6 books g - g~; 1: books (g + alpha h) - g~
+    int32_t norm;        // scale of Eq. 8: 0 l-infinity, 1 l2 (fixed summation order)
     float alpha, beta, sf;
     uint32_t key0[10];   // Philox round keys: the 64-bit seed advanced by the
     uint32_t key1[10];   // Weyl constants, one pair per round
@@ -50,12 +51,14 @@ struct BucketScale {
     int kind;       // 0 regular, 1 all levels zero, 2 non-finite (accumulator kept)
 };
 
-__device__ __forceinline__ BucketScale bucket_scale(uint32_t sbits, float sf) {
+// sbits: sign-cleared bit pattern of the bucket's max |v| (l-infinity) or of its sum of
+// squares (l2).
+__device__ __forceinline__ BucketScale bucket_scale(uint32_t sbits, float sf, int norm = 0) {
     BucketScale b;
     b.inv = 0.f; b.a = 0.f; b.scale = 0.f; b.kind = 0;
     if (sbits >= 0x7F800000u) { b.kind = 2; return b; }
-    const float scale = __uint_as_float(sbits);
     if (sbits == 0u) { b.kind = 1; return b; }
+    const float scale = norm ? __fsqrt_rn(__uint_as_float(sbits)) : __uint_as_float(sbits);
     b.inv = __fdiv_rn(sf, scale);
     if (__float_as_uint(b.inv) >= 0x7F800000u) { b.kind = 1; b.inv = 0.f; return b; }
     b.a = __fdiv_rn(scale, sf);

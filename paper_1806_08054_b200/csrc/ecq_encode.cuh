@@ -13,11 +13,13 @@ namespace ecq {
 // one hits L1/L2).  Serves bucket sizes the tiled kernel does not take (not a
 // power of two, or above 4096) and the ragged end of a vector.
 // ===========================================================================
+constexpr uint32_t kMaxL2Runs = 1024;       // any-shape path: l2 buckets of up to 32768 entries
+
 template <int NT>
 __device__ void encode_bucket_generic(const CodecParams& P, uint64_t b, uint32_t worker,
                                       uint32_t step, const float* __restrict__ g, float* h,
                                       uint32_t* __restrict__ codes, float* __restrict__ scales,
-                                      uint32_t* status, uint32_t* s_red, int tid) {
+                                      uint32_t* status, uint32_t* s_red, float* s_runs, int tid) {
     const uint64_t lo = b * (uint64_t)P.bucket;
     const uint64_t hi = (lo + P.bucket < P.d) ? lo + P.bucket : P.d;
     const uint32_t n = (uint32_t)(hi - lo);
@@ -46,7 +48,34 @@ __device__ void encode_bucket_generic(const CodecParams& P, uint64_t b, uint32_t
     m = 0;
 #pragma unroll
     for (int w = 0; w < NT / 32; ++w) m = max(m, s_red[w]);
-    const BucketScale bs = bucket_scale(m, P.sf);
+    if (P.norm == 1 && m < 0x7F800000u) {
+        // l2 scale in the stated order: every run of 32 entries front to back with one fma
+        // per entry, then the run sums pairwise in index order, level by level (ping-pong
+        // between the two halves of s_runs; at most kMaxL2Runs runs)
+        const uint32_t n_runs = (n + 31) >> 5;
+        for (uint32_t run = tid; run < n_runs; run += NT) {
+            float acc = 0.f;
+            const uint32_t e0 = run * 32, e1 = min(n, e0 + 32);
+            for (uint32_t j = e0; j < e1; ++j) {
+                const float v = __fmaf_rn(P.alpha, hb[j], gb[j]);
+                acc = __fmaf_rn(v, v, acc);
+            }
+            s_runs[run] = acc;
+        }
+        __syncthreads();
+        uint32_t cnt = n_runs, src = 0;
+        while (cnt > 1) {
+            const uint32_t up = (cnt + 1) >> 1, dst = src ^ kMaxL2Runs;
+            for (uint32_t k = tid; k < up; k += NT)
+                s_runs[dst + k] = (2 * k + 1 < cnt) ? __fadd_rn(s_runs[src + 2 * k], s_runs[src + 2 * k + 1])
+                                                    : s_runs[src + 2 * k];
+            __syncthreads();
+            cnt = up; src = dst;
+        }
+        m = __float_as_uint(s_runs[src]) & 0x7FFFFFFFu;
+        __syncthreads();
+    }
+    const BucketScale bs = bucket_scale(m, P.sf, P.norm);
     if (tid == 0) {
         scales[b] = bs.scale;
         if (bs.kind == 2) atomicOr(status, kStatusNonFinite);
@@ -110,9 +139,10 @@ encode_generic_kernel(CodecParams P, uint32_t worker, uint32_t step, const float
                       float* h, uint32_t* __restrict__ codes, float* __restrict__ scales,
                       uint32_t* status, uint64_t first_bucket, uint64_t n_buckets) {
     __shared__ uint32_t s_red[NT / 32];
+    __shared__ float s_runs[2 * kMaxL2Runs];
     for (uint64_t b = blockIdx.x; b < n_buckets; b += gridDim.x)
         encode_bucket_generic<NT>(P, first_bucket + b, worker, step, g, h, codes, scales, status,
-                                  s_red, threadIdx.x);
+                                  s_red, s_runs, threadIdx.x);
 }
 
 // ===========================================================================
@@ -230,27 +260,54 @@ encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
             G[c] = *reinterpret_cast<const float4*>(g_row + off);
             H[c] = *reinterpret_cast<const float4*>(h_row + off);
         }
-        // row max of |g + alpha h| (NaN-propagating), then over the rows of the bucket
-        float mf = 0.f;
+        // Eq. 8 scale.  l-infinity: row max of |g + alpha h| (NaN-propagating), then the max
+        // over the rows of the bucket.  l2: the row's sum of squares front to back with one
+        // fma per entry, then the row sums pairwise in index order (the xor butterfly is that
+        // tree, and addition commutes).  Both travel as sign-cleared bit patterns.
+        uint32_t m;
+        if (P.norm == 0) {
+            float mf = 0.f;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            float v0, v1, v2, v3;
-            unpack2(fma2(alpha2, pack2(H[c].x, H[c].y), pack2(G[c].x, G[c].y)), v0, v1);
-            unpack2(fma2(alpha2, pack2(H[c].z, H[c].w), pack2(G[c].z, G[c].w)), v2, v3);
-            mf = max3_abs_nan(mf, v0, v1);
-            mf = max3_abs_nan(mf, v2, v3);
+            for (int c = 0; c < 8; ++c) {
+                float v0, v1, v2, v3;
+                unpack2(fma2(alpha2, pack2(H[c].x, H[c].y), pack2(G[c].x, G[c].y)), v0, v1);
+                unpack2(fma2(alpha2, pack2(H[c].z, H[c].w), pack2(G[c].z, G[c].w)), v2, v3);
+                mf = max3_abs_nan(mf, v0, v1);
+                mf = max3_abs_nan(mf, v2, v3);
+            }
+            // non-negative floats and NaN (0x7FFFFFFF) order like their bit patterns
+            m = __float_as_uint(mf) & 0x7FFFFFFFu;
+            for (uint32_t o = 1; o < rpb && o < 32; o <<= 1)
+                m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        } else {
+            float ss = 0.f;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                float v0, v1, v2, v3;
+                unpack2(fma2(alpha2, pack2(H[c].x, H[c].y), pack2(G[c].x, G[c].y)), v0, v1);
+                unpack2(fma2(alpha2, pack2(H[c].z, H[c].w), pack2(G[c].z, G[c].w)), v2, v3);
+                ss = __fmaf_rn(v0, v0, ss); ss = __fmaf_rn(v1, v1, ss);
+                ss = __fmaf_rn(v2, v2, ss); ss = __fmaf_rn(v3, v3, ss);
+            }
+            for (uint32_t o = 1; o < rpb && o < 32; o <<= 1)
+                ss = __fadd_rn(ss, __shfl_xor_sync(0xFFFFFFFFu, ss, o));
+            m = __float_as_uint(ss);
         }
-        // non-negative floats and NaN (0x7FFFFFFF) order like their bit patterns
-        uint32_t m = __float_as_uint(mf) & 0x7FFFFFFFu;
-        for (uint32_t o = 1; o < rpb && o < 32; o <<= 1)
-            m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
         if (rpb > 32 && lane == 0) s_wmax[warp] = m;
         __syncthreads();                                   // the load buffer is free
         if (*s_abort) break;                               // uniform: set before the barrier
         if (tid == 0 && T + gridDim.x < total_tiles) issue_load(T + gridDim.x);
-        if (rpb == 64) m = max(s_wmax[warp & ~1], s_wmax[warp | 1]);
-        if (rpb == 128) m = max(max(s_wmax[0], s_wmax[1]), max(s_wmax[2], s_wmax[3]));
-        const BucketScale bs = bucket_scale(m, P.sf);
+        if (P.norm == 0) {
+            if (rpb == 64) m = max(s_wmax[warp & ~1], s_wmax[warp | 1]);
+            if (rpb == 128) m = max(max(s_wmax[0], s_wmax[1]), max(s_wmax[2], s_wmax[3]));
+        } else {
+            const float* wf = reinterpret_cast<const float*>(s_wmax);
+            float ss = __uint_as_float(m);
+            if (rpb == 64) ss = __fadd_rn(wf[warp & ~1], wf[warp | 1]);
+            if (rpb == 128) ss = __fadd_rn(__fadd_rn(wf[0], wf[1]), __fadd_rn(wf[2], wf[3]));
+            m = __float_as_uint(ss) & 0x7FFFFFFFu;
+        }
+        const BucketScale bs = bucket_scale(m, P.sf, P.norm);
         if ((tid & (rpb - 1)) == 0) {
             bt.scales[entry][(uint64_t)tile * buckets_per_tile + tid / rpb] = bs.scale;
             if (bs.kind == 2) atomicOr(status, kStatusNonFinite);
@@ -384,11 +441,12 @@ encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
     const uint64_t nb_total = (P.d + P.bucket - 1) / P.bucket;
     const uint64_t n_tail = nb_total - tail_first;
     uint32_t* s_red = reinterpret_cast<uint32_t*>(sm);   // the buffers are idle now
+    float* s_runs = reinterpret_cast<float*>(sm + 64);
     for (uint64_t k = gridDim.x - 1 - blockIdx.x; k < n_tail * n_workers; k += gridDim.x) {
         const uint32_t e = (uint32_t)(k / n_tail);
         encode_bucket_generic<kEncodeThreads>(P, tail_first + (k - e * n_tail), worker_base + e, step,
                                               bt.g[e], bt.h[e], bt.codes[e], bt.scales[e], status,
-                                              s_red, tid);
+                                              s_red, s_runs, tid);
     }
 }
 

@@ -27,11 +27,13 @@ def close(x: np.ndarray, y: np.ndarray) -> bool:
 class GpuCodec:
     """Owns a context and the per-worker device buffers of one configuration."""
 
-    def __init__(self, d, bucket, s, alpha, beta, seed, W, mode=0):
+    def __init__(self, d, bucket, s, alpha, beta, seed, W, mode=0, norm=0):
         self.d, self.bucket, self.s, self.W = d, bucket, s, W
         self.ctx = ecq.ecq_create(d, bucket, s, alpha, beta, seed)
         if mode:
             ecq.ecq_set_error_mode(self.ctx, mode)
+        if norm:
+            ecq.ecq_set_norm(self.ctx, norm)
         self.r = ecq.ecq_code_bits(self.ctx)
         self.nb = ecq.ecq_num_buckets(self.ctx)
         self.nw = ecq.ecq_codes_words(self.ctx)
@@ -84,12 +86,12 @@ def codes_np(t: torch.Tensor) -> np.ndarray:
 
 
 def full_parity(d, bucket, s, alpha, beta, seed, W, steps, grad_fn, mode=0, err0=None,
-                expect_status=ecq.ECQ_OK, check_decode=True, batch=False):
+                expect_status=ecq.ECQ_OK, check_decode=True, batch=False, norm=0):
     """Element-by-element comparison over whole vectors.
 
     ``grad_fn(worker, step)`` returns a float32 CUDA tensor of d entries.
     """
-    gpu = GpuCodec(d, bucket, s, alpha, beta, seed, W, mode)
+    gpu = GpuCodec(d, bucket, s, alpha, beta, seed, W, mode, norm)
     try:
         h_or = [np.zeros(d, np.float32) for _ in range(W)]
         if err0 is not None:
@@ -111,7 +113,7 @@ def full_parity(d, bucket, s, alpha, beta, seed, W, steps, grad_fn, mode=0, err0
 
             def one(w):
                 return oracle.encode(g_host[w], h_or[w], bucket=bucket, s=s, alpha=alpha,
-                                     beta=beta, seed=seed, worker=w, step=t, mode=mode)
+                                     beta=beta, seed=seed, worker=w, step=t, mode=mode, norm=norm)
             with ThreadPoolExecutor(max_workers=min(W, 8)) as ex:
                 res = list(ex.map(one, range(W)))
             for w in range(W):
@@ -153,9 +155,9 @@ def sample_ranges(d: int, bucket: int, span: int = 1 << 16, count: int = 3,
 class SampledOracle:
     """Follows the oracle on sampled whole-bucket ranges of a large vector."""
 
-    def __init__(self, d, bucket, s, alpha, beta, seed, W, ranges, mode=0):
+    def __init__(self, d, bucket, s, alpha, beta, seed, W, ranges, mode=0, norm=0):
         self.d, self.bucket, self.s, self.W = d, bucket, s, W
-        self.alpha, self.beta, self.seed, self.mode = alpha, beta, seed, mode
+        self.alpha, self.beta, self.seed, self.mode, self.norm = alpha, beta, seed, mode, norm
         self.ranges = ranges
         self.r = oracle.code_bits(s)
         self.h = [[np.zeros(hi - lo, np.float32) for (lo, hi) in ranges] for _ in range(W)]
@@ -166,7 +168,8 @@ class SampledOracle:
             g = grad[lo:hi].cpu().numpy()
             c_or, s_or, _ = oracle.encode(g, self.h[w][k], bucket=self.bucket, s=self.s,
                                           alpha=self.alpha, beta=self.beta, seed=self.seed,
-                                          worker=w, step=step, mode=self.mode, first_index=lo)
+                                          worker=w, step=step, mode=self.mode, first_index=lo,
+                                          norm=self.norm)
             self.msgs[w][k] = (c_or, s_or)
             w0 = lo * self.r // 32
             c_gpu = codes_np(gpu.codes[w][1][w0:w0 + c_or.size])

@@ -177,6 +177,60 @@ def test_code_histogram_and_entropy(bucket, s, d):
     gpu.close()
 
 
+# ------------------------------------------------------------ l2-norm scale ---
+@pytest.mark.parametrize("bucket", [32, 128, 512, 2048, 4096, 96, 8192, 32768])
+@pytest.mark.parametrize("s", [1, 4, 8, 128])
+def test_l2_scale_small_shapes(bucket, s):
+    for d in sorted({1, 33, bucket - 1, bucket + 1, 4096, 3 * 4096 + 5 * 32 + 7, 9 * 4096 + bucket + 40}):
+        full_parity(d, bucket, s, 1.0, 0.9, SEED, W=2, steps=2, grad_fn=randn_fn(d, base=d), norm=1,
+                    batch=(s == 4))
+
+
+def test_l2_scale_degenerate_and_wide_range_buckets():
+    B = 512
+    d = 4096 * 2 + 3 * B + 11
+    gen = torch.Generator(device="cuda"); gen.manual_seed(6)
+    g = torch.randn(d, generator=gen, device="cuda") * torch.pow(
+        10.0, torch.empty(d, device="cuda").uniform_(-4, 2, generator=gen))
+    h0 = 0.1 * torch.randn(d, generator=gen, device="cuda")
+    g[0:B] = 0; h0[0:B] = 0                          # all-zero bucket
+    g[B:2 * B] = 1e-25; h0[B:2 * B] = 0              # squares underflow to zero
+    g[2 * B:3 * B] = 0; h0[2 * B:3 * B] = 0; g[2 * B + 7] = -2.5      # a single entry
+    full_parity(d, B, 4, 1.0, 0.9, SEED, W=1, steps=2, grad_fn=lambda w, t: g, err0=[h0], norm=1)
+    g[4096 + 5] = 3e19                                 # the sum of squares overflows
+    full_parity(d, B, 4, 1.0, 0.9, SEED, W=1, steps=1, grad_fn=lambda w, t: g, err0=[h0], norm=1,
+                expect_status=ecq.ECQ_ERR_NONFINITE)
+
+
+def test_l2_scale_limits_of_the_any_shape_path():
+    ctx = ecq.ecq_create(1 << 20, 65536, 4, 1.0, 0.9, 1)
+    with pytest.raises(ecq.EcqError):
+        ecq.ecq_set_norm(ctx, 1)
+    with pytest.raises(ecq.EcqError):
+        ecq.ecq_set_norm(ctx, 2)
+    ecq.ecq_set_norm(ctx, 0)
+    ecq.ecq_destroy(ctx)
+
+
+def test_l2_scale_on_resnet50_with_the_papers_cifar_setting():
+    # bucket 4096, l2 scale, s = 4, alpha = 0.01, beta = 1.0 (the paper's CIFAR-10 footnote)
+    base = wl.WORKLOADS["resnet50"]
+    w = wl.Workload(base.name, base.index, 4, base.d, 4096, 4, 0.01, 1.0, 2, base.kind, base.layers)
+    ranges = sample_ranges(w.d, w.bucket, seed=9)
+    gpu = GpuCodec(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, w.W, norm=1)
+    so = SampledOracle(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, w.W, ranges, norm=1)
+    for t in range(w.steps):
+        gs = [wl.gradient(w, p, t, "cuda") for p in range(w.W)]
+        gpu.encode_batch(t, gs)
+        for p in range(w.W):
+            so.encode_and_compare(gpu, p, t, gs[p])
+        gpu.decode(w.W)
+        assert gpu.status() == ecq.ECQ_OK
+        so.decode_and_compare(gpu)
+    gpu.check_guards()
+    gpu.close()
+
+
 def test_argument_errors():
     with pytest.raises(ecq.EcqError):
         ecq.ecq_create(0, 512, 4, 1.0, 0.9, 1)

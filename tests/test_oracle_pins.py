@@ -442,3 +442,89 @@ def test_code_histogram_and_entropy_bound():
     assert oracle.entropy_bound_bits(np.array([256] * 8, np.uint64)) == 8 * 256 * 3.0
     assert oracle.entropy_bound_bits(np.array([0, 12345, 0], np.uint64)) == 0.0
     assert oracle.entropy_bound_bits(np.array([10, 980, 10], np.uint64)) < 1000 * 2
+
+
+# ------------------------------------------------------- l2-norm scale -------
+def _parse_positions(txt, cast):
+    pos, out = 0, {}
+    for tok in txt.split(","):
+        tok = tok.strip()
+        if tok.startswith("@"):
+            pos = int(tok[1:])
+        else:
+            out[pos] = cast(tok); pos += 1
+    return out
+
+
+def test_l2_scale_golden():
+    for row in _rows("l2_scale_cases.txt"):
+        s, B, vals, scale, levels = [x.strip() for x in row.split("|")]
+        s, B = int(s), int(B)
+        g = np.zeros(B, np.float32)
+        for k, v in _parse_positions(vals, float).items():
+            g[k] = v
+        codes, scales, st = enc(g, np.zeros(B, np.float32), bucket=B, s=s, norm=1)
+        q = oracle.unpack_levels(codes, n=B, s=s)
+        want = np.zeros(B, np.int64)
+        for k, v in _parse_positions(levels, int).items():
+            want[k] = v
+        assert st == 0 and scales[0] == np.float32(scale) and np.array_equal(q, want)
+
+
+def test_l2_scale_against_fp64_and_its_invariants():
+    rng = np.random.default_rng(51)
+    n, B, s = 5 * 512 + 100, 512, 4
+    g = (rng.standard_normal(n) * 0.01).astype(np.float32)
+    h = (rng.standard_normal(n) * 0.003).astype(np.float32)
+    v = np.float32(g + h)                                # alpha = 1: one rounded sum
+    codes, scales, st = enc(g, h.copy(), bucket=B, s=s, norm=1)
+    q = oracle.unpack_levels(codes, n=n, s=s)
+    for b in range(-(-n // B)):
+        vb = v[b * B:(b + 1) * B].astype(np.float64)
+        ref = np.sqrt((vb * vb).sum())                   # library norm in fp64
+        assert abs(float(scales[b]) - ref) <= 2.0 ** -21 * ref
+        a = float(scales[b]) / s
+        sl = slice(b * B, min((b + 1) * B, n))
+        assert np.all(np.abs(q[sl] * a - v[sl]) <= a * (1 + 2.0 ** -20))     # one level step
+        assert np.all(q[sl] * v[sl] >= 0)
+    # the l2 norm dominates the l-infinity norm, so levels sit lower than with norm = 0
+    c0, s0, _ = enc(g, h.copy(), bucket=B, s=s, norm=0)
+    assert np.all(scales >= s0) and np.abs(q).sum() < np.abs(oracle.unpack_levels(c0, n=n, s=s)).sum()
+
+
+def test_l2_quantiser_is_qsgd_lemma1():
+    # with the l2 scale the quantiser is QSGD's: unbiased, and
+    # E||eps||^2 <= min(d/s^2, sqrt(d)/s) ||v||^2  (Lemma 1)
+    rng = np.random.default_rng(61)
+    d, N = 256, 1500
+    g = (rng.standard_normal(d)).astype(np.float32)
+    for s in (1, 4, 16):
+        acc = np.zeros(d); err2 = 0.0
+        for k in range(N):
+            codes, scales, _ = enc(g, np.zeros(d, np.float32), bucket=d, s=s, norm=1, seed=k, step=k % 5)
+            gq = oracle.unpack_levels(codes, n=d, s=s) * (float(scales[0]) / s)
+            acc += gq; err2 += ((gq - g) ** 2).sum()
+        norm2 = float((g.astype(np.float64) ** 2).sum())
+        bound = min(d / s ** 2, np.sqrt(d) / s) * norm2
+        assert err2 / N <= bound
+        a = float(scales[0]) / s
+        assert np.all(np.abs(acc / N - g) <= 5 * a / (2 * np.sqrt(N)))
+
+
+def test_l2_summation_order_is_the_stated_one():
+    # integers up to 2^12 keep every partial sum exact in fp32 (< 2^24 * ...): any order gives
+    # the same sum; with wide-ranging values the stated order is reproduced step by step here
+    rng = np.random.default_rng(71)
+    B = 32 * 5                                            # five runs: the odd one is carried up
+    v = (rng.standard_normal(B) * 10.0 ** rng.uniform(-3, 3, B)).astype(np.float32)
+    runs = []
+    for r0 in range(0, B, 32):
+        acc = np.float32(0)
+        for x in v[r0:r0 + 32]:
+            acc = np.float32(np.float64(x) * np.float64(x) + np.float64(acc))    # fma: one rounding
+        runs.append(acc)
+    while len(runs) > 1:
+        runs = [np.float32(runs[k] + runs[k + 1]) if k + 1 < len(runs) else runs[k]
+                for k in range(0, len(runs), 2)]
+    _, scales, _ = enc(v, np.zeros(B, np.float32), bucket=B, s=4, norm=1)
+    assert scales[0] == np.sqrt(runs[0], dtype=np.float32)
