@@ -516,15 +516,16 @@ def test_l2_summation_order_is_the_stated_one():
     # the same sum; with wide-ranging values the stated order is reproduced step by step here
     rng = np.random.default_rng(71)
     B = 32 * 5                                            # five runs: the odd one is carried up
-    v = (rng.standard_normal(B) * 10.0 ** rng.uniform(-3, 3, B)).astype(np.float32)
-    runs = []
-    for r0 in range(0, B, 32):
-        acc = np.float32(0)
-        for x in v[r0:r0 + 32]:
-            acc = np.float32(np.float64(x) * np.float64(x) + np.float64(acc))    # fma: one rounding
-        runs.append(acc)
-    while len(runs) > 1:
-        runs = [np.float32(runs[k] + runs[k + 1]) if k + 1 < len(runs) else runs[k]
-                for k in range(0, len(runs), 2)]
-    _, scales, _ = enc(v, np.zeros(B, np.float32), bucket=B, s=4, norm=1)
-    assert scales[0] == np.sqrt(runs[0], dtype=np.float32)
+    for trial in range(40):
+        v = (rng.standard_normal(B) * 10.0 ** rng.uniform(-3, 3, B)).astype(np.float32)
+        runs = []
+        for r0 in range(0, B, 32):
+            acc = np.float32(0)
+            for x in v[r0:r0 + 32]:
+                acc = np.float32(np.float64(x) * np.float64(x) + np.float64(acc))    # fma: one rounding
+            runs.append(acc)
+        while len(runs) > 1:
+            runs = [np.float32(runs[k] + runs[k + 1]) if k + 1 < len(runs) else runs[k]
+                    for k in range(0, len(runs), 2)]
+        _, scales, _ = enc(v, np.zeros(B, np.float32), bucket=B, s=4, norm=1)
+        assert scales[0] == np.sqrt(runs[0], dtype=np.float32), trial
