@@ -75,6 +75,10 @@ bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
     if (e.base == base && e.rows == rows) { *tm = e.map; return true; }
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return false;
+    // the encoder is a driver call: a host thread that has made no runtime call yet has no
+    // context bound, so bind the current device's primary context once per thread
+    thread_local bool context_bound = false;
+    if (!context_bound) { cudaFree(nullptr); context_bound = true; }
     const cuuint64_t dims[2] = {32, rows};
     const cuuint64_t strides[1] = {128};
     const cuuint32_t box[2] = {32, (cuuint32_t)kTileRows};

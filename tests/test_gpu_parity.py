@@ -231,6 +231,42 @@ def test_l2_scale_on_resnet50_with_the_papers_cifar_setting():
     gpu.close()
 
 
+def test_one_context_from_two_host_threads_on_two_streams():
+    # a context is immutable: concurrent encodes of different workers on different streams
+    # give what serial calls give
+    import threading
+    d, B, s, W = 4096 * 40 + 72, 512, 4, 4
+    fn = randn_fn(d, base=31)
+    grads = [fn(w, 0) for w in range(W)]
+    ref = GpuCodec(d, B, s, 1.0, 0.9, SEED, W)
+    for w in range(W):
+        ref.encode(w, 0, grads[w])
+    par = GpuCodec(d, B, s, 1.0, 0.9, SEED, W)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+
+    def work(k):
+        for rep in range(20):
+            for w in range(k, W, 2):
+                if rep:
+                    par.err[w][1].zero_()
+                ecq.ecq_encode(par.ctx, w, 0, grads[w], par.err[w][1], par.codes[w][1],
+                               par.scales[w][1], stream=streams[k])
+        streams[k].synchronize()
+
+    def zeroing_stream(k):
+        with torch.cuda.stream(streams[k]):
+            work(k)
+    ts = [threading.Thread(target=zeroing_stream, args=(k,)) for k in range(2)]
+    [t.start() for t in ts]; [t.join() for t in ts]
+    torch.cuda.synchronize()
+    assert par.status() == ecq.ECQ_OK
+    for w in range(W):
+        assert torch.equal(par.codes[w][1], ref.codes[w][1]) and torch.equal(par.err[w][1], ref.err[w][1])
+        assert torch.equal(par.scales[w][1], ref.scales[w][1])
+    ref.close(); par.close()
+
+
 def test_argument_errors():
     with pytest.raises(ecq.EcqError):
         ecq.ecq_create(0, 512, 4, 1.0, 0.9, 1)
