@@ -42,7 +42,7 @@ NOMINAL_HBM_GBS = 8000.0
 # (dram__bytes_read.sum + dram__bytes_write.sum over 817,825,024 entries; see
 # profiles/encode_tiled_kernel_resnet50.md), keyed by (bucket, levels).  Traffic grows in
 # proportion to the entries of a launch.  Set an entry to None when the kernel changes.
-NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): 10192464896 / 817825024}
+NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): None}
 
 
 def code_bits(s: int) -> int:

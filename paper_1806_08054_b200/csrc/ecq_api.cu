@@ -62,17 +62,17 @@ struct ecq_ctx {
 
 namespace {
 
-// One row of the tiled view is 32 floats; a box is a whole tile of 128 rows.  A map is a
+// One row of the tiled view is 32 floats; a box is a whole tile (128 or 256 rows).  A map is a
 // pure function of (base, rows), and encoding one costs microseconds on the host, which
 // would dominate small vectors: each host thread keeps the maps it made in a small
 // direct-mapped cache.
-bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
-    struct Entry { const float* base; uint64_t rows; CUtensorMap map; };
+bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows, uint32_t box_rows) {
+    struct Entry { const float* base; uint64_t rows; uint32_t box_rows; CUtensorMap map; };
     constexpr unsigned kEntries = 256;
     thread_local Entry cache[kEntries];          // zero-initialised: base == nullptr is empty
     const uintptr_t a = reinterpret_cast<uintptr_t>(base);
-    Entry& e = cache[((a >> 8) ^ (a >> 16) ^ (a >> 24)) & (kEntries - 1)];
-    if (e.base == base && e.rows == rows) { *tm = e.map; return true; }
+    Entry& e = cache[((a >> 8) ^ (a >> 16) ^ (a >> 24) ^ box_rows) & (kEntries - 1)];
+    if (e.base == base && e.rows == rows && e.box_rows == box_rows) { *tm = e.map; return true; }
     EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return false;
     // the encoder is a driver call: a host thread that has made no runtime call yet has no
@@ -81,13 +81,13 @@ bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows) {
     if (!context_bound) { cudaFree(nullptr); context_bound = true; }
     const cuuint64_t dims[2] = {32, rows};
     const cuuint64_t strides[1] = {128};
-    const cuuint32_t box[2] = {32, (cuuint32_t)kTileRows};
+    const cuuint32_t box[2] = {32, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides,
             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
-    e.base = base; e.rows = rows; e.map = *tm;
+    e.base = base; e.rows = rows; e.box_rows = box_rows; e.map = *tm;
     return true;
 }
 
@@ -99,29 +99,29 @@ struct WorkerBuffers {
     float* scales;
 };
 
-template <int R, bool MODE1>
+template <int R, bool MODE1, int ROWS>
 int launch_encode_tiled(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
                         const WorkerBuffers* wb, cudaStream_t st, uint32_t n_tiles) {
-    using L = EncodeSmem<R>;
+    using L = EncodeSmem<R, ROWS>;
     static std::once_flag once[16];
     static int occ[16];
     const int dev = c->device & 15;
-    auto kern = encode_tiled_kernel<R, MODE1>;
+    auto kern = encode_tiled_kernel<R, MODE1, ROWS>;
     std::call_once(once[dev], [&] {
         int o = 0;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) ==
                 cudaSuccess &&
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kEncodeThreads, L::kTotal) ==
-                cudaSuccess)
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, ROWS, L::kTotal) == cudaSuccess)
             occ[dev] = o;
     });
     if (occ[dev] <= 0) return ECQ_ERR_CUDA;
     EncodeBatch bt;
-    const uint64_t rows = (uint64_t)n_tiles * kTileRows;
+    const uint64_t rows = (uint64_t)n_tiles * ROWS;
     for (uint32_t e = 0; e < (uint32_t)kMaxBatch; ++e) {
         const uint32_t src = e < n_workers ? e : 0;       // unused entries repeat entry 0
         if (e < n_workers) {
-            if (!make_tile_map(&bt.tm_g[e], wb[e].g, rows) || !make_tile_map(&bt.tm_h[e], wb[e].h, rows))
+            if (!make_tile_map(&bt.tm_g[e], wb[e].g, rows, ROWS) ||
+                !make_tile_map(&bt.tm_h[e], wb[e].h, rows, ROWS))
                 return ECQ_ERR_CUDA;
         } else {
             bt.tm_g[e] = bt.tm_g[0];
@@ -133,17 +133,30 @@ int launch_encode_tiled(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, ui
     const uint64_t total = (uint64_t)n_tiles * n_workers;
     uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
     if (grid > total) grid = (uint32_t)total;
-    kern<<<grid, kEncodeThreads, L::kTotal, st>>>(bt, c->P, worker_base, n_workers, step,
-                                                  c->d_status, n_tiles);
+    kern<<<grid, ROWS, L::kTotal, st>>>(bt, c->P, worker_base, n_workers, step, c->d_status, n_tiles);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
 }
 
+// Launches whose algorithmic traffic exceeds this run long enough (about 5 ms) to meet the
+// board's power cap, where the 128-row shape sustains more; below it the 256-row shape wins.
+constexpr uint64_t kLongLaunchBytes = 32ull << 30;
+
 template <int R>
 int launch_encode_tiled_mode(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
-                             const WorkerBuffers* wb, cudaStream_t st, uint32_t n_tiles) {
-    return c->P.mode ? launch_encode_tiled<R, true>(c, worker_base, n_workers, step, wb, st, n_tiles)
-                     : launch_encode_tiled<R, false>(c, worker_base, n_workers, step, wb, st, n_tiles);
+                             const WorkerBuffers* wb, cudaStream_t st) {
+    const uint64_t bytes = (uint64_t)n_workers * c->P.d * 12;
+    const bool small_tiles = bytes > kLongLaunchBytes || c->P.d < 8192;
+    const uint64_t elems = small_tiles ? 4096 : 8192;
+    const uint64_t n_tiles64 = c->P.d / elems;
+    if (n_tiles64 == 0 || n_tiles64 * n_workers > 0xFFFFFFFFull || n_tiles64 * 256 > 0x7FFFFFFFull)
+        return -1;                                        // not for the tiled path
+    const uint32_t n_tiles = (uint32_t)n_tiles64;
+    if (small_tiles)
+        return c->P.mode ? launch_encode_tiled<R, true, 128>(c, worker_base, n_workers, step, wb, st, n_tiles)
+                         : launch_encode_tiled<R, false, 128>(c, worker_base, n_workers, step, wb, st, n_tiles);
+    return c->P.mode ? launch_encode_tiled<R, true, 256>(c, worker_base, n_workers, step, wb, st, n_tiles)
+                     : launch_encode_tiled<R, false, 256>(c, worker_base, n_workers, step, wb, st, n_tiles);
 }
 
 int launch_encode_generic(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, float* h,
@@ -160,20 +173,20 @@ int launch_encode_generic(ecq_ctx* c, uint32_t worker, uint32_t step, const floa
 // path takes the whole batch in one launch; other shapes go one launch per worker.
 int encode_batch_impl(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
                       const WorkerBuffers* wb, cudaStream_t st) {
-    const uint64_t n_tiles64 = c->tiled_ok ? c->P.d / kTileElems : 0;
-    if (n_tiles64 > 0 && n_tiles64 * n_workers <= 0xFFFFFFFFull && n_tiles64 * kTileRows <= 0x7FFFFFFFull) {
-        const uint32_t n_tiles = (uint32_t)n_tiles64;
+    if (c->tiled_ok) {
+        int rc = -1;
         switch (c->P.r) {
-            case 2: return launch_encode_tiled_mode<2>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 3: return launch_encode_tiled_mode<3>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 4: return launch_encode_tiled_mode<4>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 5: return launch_encode_tiled_mode<5>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 6: return launch_encode_tiled_mode<6>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 7: return launch_encode_tiled_mode<7>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 8: return launch_encode_tiled_mode<8>(c, worker_base, n_workers, step, wb, st, n_tiles);
-            case 9: return launch_encode_tiled_mode<9>(c, worker_base, n_workers, step, wb, st, n_tiles);
+            case 2: rc = launch_encode_tiled_mode<2>(c, worker_base, n_workers, step, wb, st); break;
+            case 3: rc = launch_encode_tiled_mode<3>(c, worker_base, n_workers, step, wb, st); break;
+            case 4: rc = launch_encode_tiled_mode<4>(c, worker_base, n_workers, step, wb, st); break;
+            case 5: rc = launch_encode_tiled_mode<5>(c, worker_base, n_workers, step, wb, st); break;
+            case 6: rc = launch_encode_tiled_mode<6>(c, worker_base, n_workers, step, wb, st); break;
+            case 7: rc = launch_encode_tiled_mode<7>(c, worker_base, n_workers, step, wb, st); break;
+            case 8: rc = launch_encode_tiled_mode<8>(c, worker_base, n_workers, step, wb, st); break;
+            case 9: rc = launch_encode_tiled_mode<9>(c, worker_base, n_workers, step, wb, st); break;
             default: break;
         }
+        if (rc >= 0) return rc;
     }
     for (uint32_t e = 0; e < n_workers; ++e) {
         const int rc = launch_encode_generic(c, worker_base + e, step, wb[e].g, wb[e].h, wb[e].codes,
