@@ -38,11 +38,12 @@ METRIC = "codec_step_throughput"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes per entry of the batched tiled encode kernel from an ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum over 817,825,024 entries; see
-# profiles/encode_tiled_kernel_resnet50.md), keyed by (bucket, levels).  Traffic grows in
-# proportion to the entries of a launch.  Set an entry to None when the kernel changes.
-NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): None}
+# DRAM bytes per entry of the batched tiled encode kernel from an ncu capture of the default
+# workload's own launch (dram__bytes_read.sum + dram__bytes_write.sum = 141,431,158,016 bytes
+# over 11,310,497,792 entries; see profiles/encode_tiled_kernel.md), keyed by (bucket, levels).
+# Traffic grows in proportion to the entries of a launch.  Set an entry to None when the
+# kernel changes.
+NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): 141431158016 / 11310497792}
 
 
 def code_bits(s: int) -> int:
