@@ -1,0 +1,51 @@
+"""The benchmark's JSON line, on a small workload: every key of the contract is present and
+consistent (own arm and reference arm)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _run(*extra):
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *extra],
+                         capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-3000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1, "exactly one JSON line expected"
+    return json.loads(lines[0])
+
+
+def test_own_arm_line():
+    j = _run("--workload", "lsq_4m", "--steps", "3", "--warmup", "3", "--cpu-elems", "131072")
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step",
+                "higher_is_better", "scaling", "vs_baseline", "dtype", "data", "config", "roofline",
+                "cpu_baseline", "e2e", "gpu_launches", "clocks", "encode", "decode", "message"):
+        assert key in j, key
+    assert j["metric"] == "codec_step_throughput" and j["unit"] == "GB/s" and j["value"] > 0
+    assert j["n_gpus"] == 1 and j["steps"] == 3 and j["warmup"] >= 3 and j["scaling"] == "weak"
+    assert j["vs_baseline"] is None and j["dtype"] == "f32" and j["data"] == "synthetic"
+    assert j["config"]["workload"] == "lsq_4m" and "model" not in j["config"]
+    rf = j["roofline"]
+    assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and rf["peak"] > 0
+    assert abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9
+    assert j["gpu_launches"] == 2 * 3                       # one batched encode + one decode per step
+    cb = j["cpu_baseline"]
+    assert cb["kind"] == "oracle" and cb["cores"] == 1 and cb["value"] > 0 and "sample" in cb
+    e2e = j["e2e"]
+    assert e2e["value"] > 0 and e2e["h2d_bytes_per_step"] == 8 * 4194304 * 4
+    assert e2e["d2h_bytes_per_step"] == 4194304 * 4 and e2e["value"] < j["value"]
+    assert set(j["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    m = j["message"]
+    assert m["entropy_bound_bits_per_entry"] <= m["fixed_bits_per_entry"] + 1e-9
+
+
+def test_reference_arm_line():
+    j = _run("--impl", "reference", "--workload", "lsq_4m", "--steps", "1", "--warmup", "0",
+             "--ref-elems", "65536")
+    assert j["impl"] == "reference" and j["metric"] == "codec_step_throughput" and j["value"] > 0
+    assert j["cpu_baseline"]["kind"] == "oracle" and j["e2e"]["h2d_bytes_per_step"] == 0
