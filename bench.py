@@ -359,6 +359,14 @@ def main():
                         "compression_entropy_bound": 32.0 * d / (entropy_bits + 32.0 * nb),
                         "note": "worker 0, last timed step; the paper's Table 1 ratios are "
                                 "entropy-coded on other workloads (context only)"},
+            # the decode kernel's own bound: one logic instruction per code on the ALU pipe
+            # (16 lanes per clock per SM sub-partition)
+            "decode_roofline": {"kernel": "decode_tiled_kernel", "bound": "alu",
+                                "achieved": W * d * args.steps / (dec_ms * 1e-3) / 1e12,
+                                "peak": 148 * 4 * 16 * 1.965e9 / 1e12, "unit": "Tcodes/s",
+                                "frac": (W * d * args.steps / (dec_ms * 1e-3)) / (148 * 4 * 16 * 1.965e9),
+                                "peak_source": "derived: 148 SMs x 4 x 16 lanes x 1.965 GHz, "
+                                               "1 logic op per code"},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
