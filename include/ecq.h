@@ -42,7 +42,8 @@ extern "C" {
 
 typedef struct ecq_ctx ecq_ctx;
 
-#define ECQ_MAX_WORKERS 64   /* most workers one batched or receiver-side call takes */
+#define ECQ_MAX_WORKERS 64          /* workers (messages) one kernel launch serves */
+#define ECQ_MAX_WORKERS_TOTAL 1024  /* most workers ecq_encode_batch / ecq_decode_mean[_update] take */
 
 enum {
     ECQ_OK = 0,
@@ -133,8 +134,9 @@ int ecq_encode(ecq_ctx* ctx, uint32_t worker, uint32_t step, const float* grad,
  * the loop "for p = 1..P" of phase 1, on a single GPU that holds all P workers'
  * slices).  Results are identical to W calls of ecq_encode(ctx, w, step, grads[w],
  * errs[w], codes[w], scales[w]); a single launch spares W-1 launch ramps and tails,
- * which matters for vectors of tens of megabytes.
- *   W       1..ECQ_MAX_WORKERS
+ * which matters for vectors of tens of megabytes.  Beyond ECQ_MAX_WORKERS workers there
+ * is one launch per ECQ_MAX_WORKERS of them, with the same results.
+ *   W       1..ECQ_MAX_WORKERS_TOTAL
  *   grads, errs, codes, scales   HOST arrays of W device pointers each, with the
  *           meaning, sizes and alignment of ecq_encode's arguments; read before the
  *           call returns
@@ -146,11 +148,15 @@ int ecq_encode_batch(ecq_ctx* ctx, uint32_t W, uint32_t step, const float* const
 /*
  * Receiver side (Eq. 4 and Algorithm 1, "compute global gradients"):
  *   out_i = (1/W) * sum_{w<W} q_{w,i} * (scales_w[b(i)] / s)
- *   W       number of messages, 1..ECQ_MAX_WORKERS
+ *   W       number of messages, 1..ECQ_MAX_WORKERS_TOTAL
  *   codes   HOST array of W device pointers to the workers' code streams
  *   scales  HOST array of W device pointers to the workers' scales
  *   out [d] the averaged dequantised gradient
- * The two pointer arrays are read before the call returns.
+ * The two pointer arrays are read before the call returns.  Up to ECQ_MAX_WORKERS
+ * messages are summed in one launch; beyond that there is one launch per
+ * ECQ_MAX_WORKERS messages, each continuing the sum of the previous one (kept in
+ * `out` meanwhile) in the same ascending order of w, so the result is the same
+ * chain of fp32 operations as a single pass.
  */
 int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
                     const float* const* scales, float* out, void* cuda_stream);
@@ -162,6 +168,8 @@ int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
  *   params_i <- fma(-eta, g~_i, params_i)       (one rounding)
  *   out_i    = g~_i when out is not NULL
  *   params [d]  in/out, 16-byte aligned; out [d] or NULL, must not alias params
+ *   W       as in ecq_decode_mean; with more than ECQ_MAX_WORKERS messages `out` is
+ *           required (it carries the running sum between launches; ECQ_ERR_ARG if NULL)
  * Saves the separate pass over the decoded gradient that an optimiser step would make.
  */
 int ecq_decode_mean_update(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,

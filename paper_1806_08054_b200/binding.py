@@ -19,6 +19,7 @@ ECQ_OK, ECQ_ERR_ARG, ECQ_ERR_CUDA, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT, ECQ_ERR_A
 ECQ_ERR_TOO_LARGE = 6
 ECQ_STATIC_SCRATCH_BYTES = 4 << 20
 ECQ_MAX_WORKERS = 64
+ECQ_MAX_WORKERS_TOTAL = 1024
 
 _lib = None
 

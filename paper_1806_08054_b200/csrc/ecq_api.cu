@@ -1,4 +1,5 @@
 // C ABI of the ECQ-SGD codec: argument checks, launch configuration, status word.
+#include <algorithm>
 #include <atomic>
 #include <cstdint>
 #include <cstdlib>
@@ -204,20 +205,20 @@ int encode_impl(ecq_ctx* c, uint32_t worker, uint32_t step, const float* g, floa
 
 template <int R>
 void launch_decode(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out, cudaStream_t st,
-                   float w_recip, int w_pow2) {
+                   float w_recip, int w_pow2, DecodeSlice sl) {
     constexpr int G = DecodeGroup<R>::kElems;
     const uint64_t n_groups = (c->P.d + G - 1) / G;
     uint64_t blocks = (n_groups + 255) / 256;
     const uint64_t cap = (uint64_t)c->sm_count * 64;
     if (blocks > cap) blocks = cap;
     decode_mean_kernel<R><<<(uint32_t)blocks, 256, 0, st>>>(c->P, W, tab, out, n_groups,
-                                                            c->n_words, w_recip, w_pow2);
+                                                            c->n_words, w_recip, w_pow2, sl);
 }
 
 // Tiled decode: returns false when the shape is not covered (caller falls back).
-template <int R>
+template <int R, bool CARRY>
 bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out,
-                         cudaStream_t st, float w_recip, int w_pow2) {
+                         cudaStream_t st, float w_recip, int w_pow2, DecodeSlice sl) {
     using L = DecodeTiled<R>;
     const uint32_t B = c->P.bucket;
     const uint64_t n_tiles64 = c->P.d / kDecTileElems;
@@ -228,7 +229,7 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, Decode
     static std::once_flag once[16];
     static int occ[16];
     const int dev = c->device & 15;
-    auto kern = decode_tiled_kernel<R>;
+    auto kern = decode_tiled_kernel<R, CARRY>;
     std::call_once(once[dev], [&] {
         int o = 0;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmem) ==
@@ -243,45 +244,63 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, Decode
     const uint32_t want = (n_tiles + kDecWarps - 1) / kDecWarps;
     if (grid > want) grid = want;
     kern<<<grid, kDecWarps * 32, L::kSmem, st>>>(c->P, W, tab, out, n_tiles, c->n_words, w_recip,
-                                                 w_pow2, 0x4B000000u);
+                                                 w_pow2, 0x4B000000u, sl);
     return true;
 }
 
-int decode_impl(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out, cudaStream_t st) {
-    const int w_pow2 = (W & (W - 1)) == 0;
-    const float w_recip = 1.0f / (float)W;
+// One launch over the W <= 64 messages of `tab`; w_all is the number of messages of the whole
+// mean (the divisor), of which this launch may be one slice (out.first / out.last).
+int decode_launch(ecq_ctx* c, uint32_t W, uint32_t w_all, const MessageTable& tab, DecodeOut out,
+                  bool first, bool last, cudaStream_t st) {
+    const int w_pow2 = (w_all & (w_all - 1)) == 0;
+    const float w_recip = 1.0f / (float)w_all;
+    const DecodeSlice sl{(float)w_all, first, last};
     bool done = false;
     switch (c->P.r) {
-        case 2: done = launch_decode_tiled<2>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 3: done = launch_decode_tiled<3>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 4: done = launch_decode_tiled<4>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 5: done = launch_decode_tiled<5>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 6: done = launch_decode_tiled<6>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 7: done = launch_decode_tiled<7>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 8: done = launch_decode_tiled<8>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 9: done = launch_decode_tiled<9>(c, W, tab, out, st, w_recip, w_pow2); break;
+#define ECQ_CASE(R) case R: done = (first && last)                                                      \
+            ? launch_decode_tiled<R, false>(c, W, tab, out, st, w_recip, w_pow2, sl)                     \
+            : launch_decode_tiled<R, true>(c, W, tab, out, st, w_recip, w_pow2, sl); break;
+        ECQ_CASE(2) ECQ_CASE(3) ECQ_CASE(4) ECQ_CASE(5) ECQ_CASE(6) ECQ_CASE(7) ECQ_CASE(8) ECQ_CASE(9)
+#undef ECQ_CASE
         default: break;
     }
     if (!done) switch (c->P.r) {
-        case 2: launch_decode<2>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 3: launch_decode<3>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 4: launch_decode<4>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 5: launch_decode<5>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 6: launch_decode<6>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 7: launch_decode<7>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 8: launch_decode<8>(c, W, tab, out, st, w_recip, w_pow2); break;
-        case 9: launch_decode<9>(c, W, tab, out, st, w_recip, w_pow2); break;
+#define ECQ_CASE(R) case R: launch_decode<R>(c, W, tab, out, st, w_recip, w_pow2, sl); break;
+        ECQ_CASE(2) ECQ_CASE(3) ECQ_CASE(4) ECQ_CASE(5) ECQ_CASE(6) ECQ_CASE(7) ECQ_CASE(8) ECQ_CASE(9)
+#undef ECQ_CASE
         default: {
             const uint64_t n_groups = (c->P.d + 31) / 32;
             uint64_t blocks = (n_groups + 255) / 256;
             const uint64_t cap = (uint64_t)c->sm_count * 64;
             if (blocks > cap) blocks = cap;
             decode_mean_generic_kernel<<<(uint32_t)blocks, 256, 0, st>>>(
-                c->P, W, tab, out, n_groups, c->n_words, w_recip, w_pow2);
+                c->P, W, tab, out, n_groups, c->n_words, w_recip, w_pow2, sl);
         }
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+// Eq. 4 over W messages, 64 per launch; between launches the running sums live in `out`.
+int decode_impl(ecq_ctx* c, uint32_t W, const uint32_t* const* codes, const float* const* scales,
+                float* out, float* params, float neg_eta, cudaStream_t st) {
+    if (W > (uint32_t)kMaxBatch && !out) return ECQ_ERR_ARG;
+    for (uint32_t w = 0; w < W; ++w)
+        if (!codes[w] || !scales[w] || !aligned16(codes[w]) || !aligned4(scales[w]))
+            return ECQ_ERR_ARG;
+    for (uint32_t w0 = 0; w0 < W; w0 += kMaxBatch) {
+        const uint32_t n = std::min<uint32_t>(kMaxBatch, W - w0);
+        MessageTable tab;
+        std::memset(&tab, 0, sizeof(tab));
+        for (uint32_t k = 0; k < n; ++k) {
+            tab.codes[k] = codes[w0 + k];
+            tab.scales[k] = scales[w0 + k];
+        }
+        const int rc = decode_launch(c, n, W, tab, DecodeOut{out, params, neg_eta}, w0 == 0,
+                                     w0 + n == W, st);
+        if (rc != ECQ_OK) return rc;
+    }
+    return ECQ_OK;
 }
 
 inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
@@ -373,48 +392,39 @@ int ecq_encode(ecq_ctx* c, uint32_t worker, uint32_t step, const float* grad, fl
 int ecq_encode_batch(ecq_ctx* c, uint32_t W, uint32_t step, const float* const* grads,
                      float* const* errs, uint32_t* const* codes, float* const* scales,
                      void* cuda_stream) {
-    if (!c || !grads || !errs || !codes || !scales || W == 0 || W > ECQ_MAX_WORKERS)
+    if (!c || !grads || !errs || !codes || !scales || W == 0 || W > ECQ_MAX_WORKERS_TOTAL)
         return ECQ_ERR_ARG;
-    WorkerBuffers wb[ECQ_MAX_WORKERS];
     for (uint32_t w = 0; w < W; ++w) {
         if (!grads[w] || !errs[w] || !codes[w] || !scales[w]) return ECQ_ERR_ARG;
         if (!aligned16(grads[w]) || !aligned16(errs[w]) || !aligned16(codes[w]) || !aligned4(scales[w]))
             return ECQ_ERR_ARG;
-        wb[w] = {grads[w], errs[w], codes[w], scales[w]};
     }
-    return encode_batch_impl(c, 0, W, step, wb, static_cast<cudaStream_t>(cuda_stream));
+    // one launch per ECQ_MAX_WORKERS workers
+    for (uint32_t w0 = 0; w0 < W; w0 += ECQ_MAX_WORKERS) {
+        const uint32_t n = std::min<uint32_t>(ECQ_MAX_WORKERS, W - w0);
+        WorkerBuffers wb[ECQ_MAX_WORKERS];
+        for (uint32_t k = 0; k < n; ++k)
+            wb[k] = {grads[w0 + k], errs[w0 + k], codes[w0 + k], scales[w0 + k]};
+        const int rc = encode_batch_impl(c, w0, n, step, wb, static_cast<cudaStream_t>(cuda_stream));
+        if (rc != ECQ_OK) return rc;
+    }
+    return ECQ_OK;
 }
 
 int ecq_decode_mean(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,
                     const float* const* scales, float* out, void* cuda_stream) {
-    if (!c || !codes || !scales || !out || W == 0 || W > ECQ_MAX_WORKERS) return ECQ_ERR_ARG;
+    if (!c || !codes || !scales || !out || W == 0 || W > ECQ_MAX_WORKERS_TOTAL) return ECQ_ERR_ARG;
     if (!aligned16(out)) return ECQ_ERR_ARG;
-    MessageTable tab;
-    std::memset(&tab, 0, sizeof(tab));
-    for (uint32_t w = 0; w < W; ++w) {
-        if (!codes[w] || !scales[w] || !aligned16(codes[w]) || !aligned4(scales[w]))
-            return ECQ_ERR_ARG;
-        tab.codes[w] = codes[w];
-        tab.scales[w] = scales[w];
-    }
-    return decode_impl(c, W, tab, DecodeOut{out, nullptr, 0.f}, static_cast<cudaStream_t>(cuda_stream));
+    return decode_impl(c, W, codes, scales, out, nullptr, 0.f, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int ecq_decode_mean_update(ecq_ctx* c, uint32_t W, const uint32_t* const* codes,
                            const float* const* scales, float eta, float* params, float* out,
                            void* cuda_stream) {
-    if (!c || !codes || !scales || !params || W == 0 || W > ECQ_MAX_WORKERS) return ECQ_ERR_ARG;
+    if (!c || !codes || !scales || !params || W == 0 || W > ECQ_MAX_WORKERS_TOTAL) return ECQ_ERR_ARG;
     if (!aligned16(params) || (out && !aligned16(out)) || !(eta == eta) || params == out)
         return ECQ_ERR_ARG;
-    MessageTable tab;
-    std::memset(&tab, 0, sizeof(tab));
-    for (uint32_t w = 0; w < W; ++w) {
-        if (!codes[w] || !scales[w] || !aligned16(codes[w]) || !aligned4(scales[w]))
-            return ECQ_ERR_ARG;
-        tab.codes[w] = codes[w];
-        tab.scales[w] = scales[w];
-    }
-    return decode_impl(c, W, tab, DecodeOut{out, params, -eta}, static_cast<cudaStream_t>(cuda_stream));
+    return decode_impl(c, W, codes, scales, out, params, -eta, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int ecq_code_histogram(ecq_ctx* c, const uint32_t* codes, uint64_t* counts, void* cuda_stream) {
@@ -507,7 +517,7 @@ int ecq_step_host(ecq_ctx* c, uint32_t W, uint32_t step, const float* const* gra
         rc = encode_impl(c, w, step, stage[sl], err_dev + (uint64_t)w * d, codes, scales, st);
         cudaEventRecord(c->ev_encoded[sl], st);
     }
-    if (rc == ECQ_OK) rc = decode_impl(c, W, tab, DecodeOut{out_dev, nullptr, 0.f}, st);
+    if (rc == ECQ_OK) rc = decode_launch(c, W, W, tab, DecodeOut{out_dev, nullptr, 0.f}, true, true, st);
     if (rc == ECQ_OK &&
         cudaMemcpyAsync(out_host, out_dev, d * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         rc = ECQ_ERR_CUDA;
@@ -633,7 +643,7 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
         tab.scales[w] = scales;
         rc = encode_impl(&c, w, step, grads[w], err + (uint64_t)w * d, codes, scales, st);
     }
-    if (rc == ECQ_OK) rc = decode_impl(&c, W, tab, DecodeOut{out, nullptr, 0.f}, st);
+    if (rc == ECQ_OK) rc = decode_launch(&c, W, W, tab, DecodeOut{out, nullptr, 0.f}, true, true, st);
     uint32_t bits = 0;
     if (cudaMemcpyAsync(&bits, c.d_status, sizeof(bits), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)

@@ -13,10 +13,18 @@ struct MessageTable {
 
 // Where a decoded mean goes: to `out` (may be null), and, for the fused model update of
 // Algorithm 1 ("update model parameters w <- w - eta * g~"), into `params` (may be null).
+// More than 64 messages are summed over several launches of 64: every launch but the first
+// starts from the running sums a previous one left in `out` (first == 0), and every launch
+// but the last leaves its running sums there instead of the mean (last == 0).  The chain of
+// multiply-adds is the same as in one pass.  (DecodeSlice below.)
 struct DecodeOut {
     float* out;
     float* params;
     float neg_eta;
+};
+struct DecodeSlice {
+    float w_total;      // number of messages of the whole mean (the divisor)
+    int first, last;
 };
 __device__ __forceinline__ void emit1(const DecodeOut& o, uint64_t i, float v) {
     if (o.params) o.params[i] = __fmaf_rn(o.neg_eta, v, o.params[i]);
@@ -44,7 +52,7 @@ template <int R>
 __global__ void __launch_bounds__(256)
 decode_mean_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
                    const DecodeOut dst, const uint64_t n_groups, const uint64_t n_words,
-                   const float w_recip, const int w_pow2) {
+                   const float w_recip, const int w_pow2, const DecodeSlice sl) {
     constexpr int G = DecodeGroup<R>::kElems;
     constexpr int NW = DecodeGroup<R>::kWords;
     constexpr uint32_t mask = (1u << R) - 1u;
@@ -56,7 +64,7 @@ decode_mean_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         const uint64_t w0 = gi * NW;
         float acc[G];
 #pragma unroll
-        for (int j = 0; j < G; ++j) acc[j] = 0.f;
+        for (int j = 0; j < G; ++j) acc[j] = (sl.first || i0 + j >= P.d) ? 0.f : dst.out[i0 + j];
         for (uint32_t w = 0; w < W; ++w) {
             const float a = __fdiv_rn(__ldg(tab.scales[w] + b), P.sf);
             uint32_t cw[NW + 1];
@@ -74,9 +82,15 @@ decode_mean_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
                 acc[j] = __fmaf_rn(q, a, acc[j]);
             }
         }
+        if (!sl.last) {
+#pragma unroll
+            for (int j = 0; j < G; ++j)
+                if (i0 + j < P.d) dst.out[i0 + j] = acc[j];
+            continue;
+        }
 #pragma unroll
         for (int j = 0; j < G; ++j)
-            acc[j] = w_pow2 ? __fmul_rn(acc[j], w_recip) : __fdiv_rn(acc[j], (float)W);
+            acc[j] = w_pow2 ? __fmul_rn(acc[j], w_recip) : __fdiv_rn(acc[j], sl.w_total);
         if (i0 + G <= P.d) {
 #pragma unroll
             for (int j = 0; j < G; j += 4)
@@ -94,7 +108,7 @@ __global__ void __launch_bounds__(256)
 decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
                            const __grid_constant__ MessageTable tab, const DecodeOut dst,
                            const uint64_t n_groups, const uint64_t n_words, const float w_recip,
-                           const int w_pow2) {
+                           const int w_pow2, const DecodeSlice sl) {
     const uint32_t r = P.r, mask = (1u << r) - 1u;
     const float magic = 8388608.f + (float)P.s;
     for (uint64_t gi = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; gi < n_groups;
@@ -104,7 +118,7 @@ decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
         const uint64_t w0 = gi * r;
         for (int j = 0; j < 32 && i0 + j < P.d; ++j) {
             const uint32_t bit = j * r, wi = bit >> 5, sh = bit & 31;
-            float acc = 0.f;
+            float acc = sl.first ? 0.f : dst.out[i0 + j];
             for (uint32_t w = 0; w < W; ++w) {
                 const float a = __fdiv_rn(__ldg(tab.scales[w] + b), P.sf);
                 const uint32_t lo = __ldg(tab.codes[w] + w0 + wi);
@@ -114,7 +128,8 @@ decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
                 const float q = __fsub_rn(__uint_as_float(0x4B000000u | c), magic);
                 acc = __fmaf_rn(q, a, acc);
             }
-            emit1(dst, i0 + j, w_pow2 ? __fmul_rn(acc, w_recip) : __fdiv_rn(acc, (float)W));
+            if (!sl.last) dst.out[i0 + j] = acc;
+            else emit1(dst, i0 + j, w_pow2 ? __fmul_rn(acc, w_recip) : __fdiv_rn(acc, sl.w_total));
         }
     }
 }
@@ -162,12 +177,17 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-template <int R>
+// CARRY: the launch is one slice of a longer sum (`sl` is honoured); without it the launch
+// is the whole sum over W messages.
+template <int R, bool CARRY>
 __global__ void __launch_bounds__(kDecWarps * 32)
 decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
                     const DecodeOut dst, const uint32_t n_tiles, const uint64_t n_words,
-                    const float w_recip, const int w_pow2, const uint32_t exp23_bits) {
+                    const float w_recip, const int w_pow2, const uint32_t exp23_bits,
+                    const DecodeSlice sl) {
     using L = DecodeTiled<R>;
+    const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
+    const float w_total = CARRY ? sl.w_total : (float)W;
     constexpr int D = L::kRing;
     constexpr int FIT = L::kFit;
     constexpr uint32_t mask = (1u << R) - 1u;
@@ -260,6 +280,30 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         uint64_t acc2[16];                      // outputs (2k, 2k+1) as fp32 pairs
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc2[j] = 0ull;
+        if (!first) {
+            // running sums of the earlier messages: coalesced loads, transposed through the
+            // staging buffer to one row per lane, and given the powers of two of their fields
+            const float* src = dst.out + (uint64_t)tile * kDecTileElems;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
+                *reinterpret_cast<float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4)) =
+                    *reinterpret_cast<const float4*>(src + idx * 4);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 v = *reinterpret_cast<const float4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4));
+                const float in[4] = {v.x, v.y, v.z, v.w};
+                float sc[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    sc[q] = __fmul_rn(in[q], __uint_as_float((uint32_t)(127 - 22 + ((4 * c + q) % FIT) * R) << 23));
+                acc2[2 * c] = pack2(sc[0], sc[1]);
+                acc2[2 * c + 1] = pack2(sc[2], sc[3]);
+            }
+            __syncwarp();
+        }
 
 #pragma unroll 1
         for (uint32_t w = 0; w < W; ++w) {
@@ -312,14 +356,18 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         float acc[32];
 #pragma unroll
         for (int j = 0; j < 16; ++j) unpack2(acc2[j], acc[2 * j], acc[2 * j + 1]);
-        if (w_pow2) {
+        if (!last) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                acc[j] = __fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23));
+        } else if (w_pow2) {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
                 acc[j] = __fmul_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), w_recip);
         } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-                acc[j] = __fdiv_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), (float)W);
+                acc[j] = __fdiv_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), w_total);
         }
         // transpose through the staging buffer: row-per-lane -> coalesced 16-byte stores
 #pragma unroll
@@ -332,7 +380,8 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         for (int k = 0; k < 8; ++k) {
             const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
             const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
-            emit4(dst, o + idx * 4, v);
+            if (last) emit4(dst, o + idx * 4, v);
+            else *reinterpret_cast<float4*>(dst.out + o + idx * 4) = v;
         }
         __syncwarp();
     }
@@ -345,7 +394,7 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
          i += (uint64_t)gridDim.x * blockDim.x) {
         const uint64_t b = i / P.bucket, bit = i * R, wi = bit >> 5;
         const uint32_t sh = (uint32_t)(bit & 31);
-        float acc1 = 0.f;
+        float acc1 = first ? 0.f : dst.out[i];
         for (uint32_t w = 0; w < W; ++w) {
             const float a = __fdiv_rn(__ldg(tab.scales[w] + b), P.sf);
             const uint32_t lo = __ldg(tab.codes[w] + wi);
@@ -353,7 +402,8 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
             const uint32_t c = __funnelshift_r(lo, hi1, sh) & mask;
             acc1 = __fmaf_rn(__fsub_rn(__uint_as_float(0x4B000000u | c), magic), a, acc1);
         }
-        emit1(dst, i, w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, (float)W));
+        if (!last) dst.out[i] = acc1;
+        else emit1(dst, i, w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, w_total));
     }
 }
 

@@ -123,6 +123,50 @@ def test_decode_worker_counts():
         full_parity(d, B, s, 1.0, 0.9, SEED, W=W, steps=1, grad_fn=randn_fn(d, base=W))
 
 
+@pytest.mark.parametrize("bucket,s,W,d", [(512, 4, 65, 4096 * 2 + 600), (512, 4, 128, 4096 + 36),
+                                            (2048, 1, 150, 4096 * 3 + 24), (96, 8, 70, 3001),
+                                            (128, 300, 129, 2500), (32, 2, 66, 4096 + 40),
+                                            (4096, 128, 200, 4096 * 2 + 5)])
+def test_more_workers_than_one_launch_serves(bucket, s, W, d):
+    # beyond 64 messages the receiver sums 64 per launch and carries the running sums in
+    # `out`; the sender batches 64 workers per launch.  Same chain of operations as one pass.
+    before = ecq.ecq_launch_count()
+    full_parity(d, bucket, s, 1.0, 0.9, SEED, W=W, steps=2, grad_fn=randn_fn(d, base=W), batch=True)
+    launches = ecq.ecq_launch_count() - before
+    chunks = -(-W // ecq.binding.ECQ_MAX_WORKERS)
+    tiled = (bucket & (bucket - 1)) == 0 and bucket <= 4096 and d >= 4096
+    assert launches == 2 * ((chunks if tiled else W) + chunks)
+
+
+def test_fused_model_update_with_more_workers_than_one_launch_serves():
+    d, bucket, s, W = 4096 * 2 + 77, 512, 4, 100
+    gpu = GpuCodec(d, bucket, s, 1.0, 0.9, SEED, W)
+    fn = randn_fn(d, base=11)
+    grads = [fn(w, 0) for w in range(W)]
+    gpu.encode_batch(0, grads)
+    msgs = []
+    for w in range(W):
+        h = np.zeros(d, np.float32)
+        c, sc, _ = oracle.encode(grads[w].cpu().numpy(), h, bucket=bucket, s=s, alpha=1.0, beta=0.9,
+                                 seed=SEED, worker=w, step=0)
+        msgs.append((c, sc))
+    gen = torch.Generator(device="cuda"); gen.manual_seed(3)
+    p0 = torch.randn(d, generator=gen, device="cuda")
+    params = p0.clone()
+    codes, scales = [c[1] for c in gpu.codes], [x[1] for x in gpu.scales]
+    ecq.ecq_decode_mean_update(gpu.ctx, codes, scales, 0.05, params, gpu.out[1])
+    assert gpu.status() == ecq.ECQ_OK
+    p_or = p0.cpu().numpy().copy()
+    mean = oracle.decode_mean_update([m[0] for m in msgs], [m[1] for m in msgs], p_or, eta=0.05,
+                                     bucket=bucket, s=s)
+    assert np.array_equal(params.cpu().numpy().view(np.uint32), p_or.view(np.uint32))
+    assert np.array_equal(gpu.out[1].cpu().numpy().view(np.uint32), mean.view(np.uint32))
+    gpu.check_guards()
+    with pytest.raises(ecq.EcqError):       # the running sums need `out` between launches
+        ecq.ecq_decode_mean_update(gpu.ctx, codes, scales, 0.05, params, None)
+    gpu.close()
+
+
 @pytest.mark.parametrize("bucket,s,W,d", [(512, 4, 4, 4096 * 5 + 700), (2048, 1, 16, 4096 * 3 + 2048 + 24),
                                             (96, 8, 3, 5000), (128, 300, 2, 3000), (512, 8, 8, 777)])
 def test_fused_model_update(bucket, s, W, d):
@@ -283,7 +327,7 @@ def test_argument_errors():
                        gpu.scales[0][1])
     L = ecq.binding.lib()
     assert L.ecq_decode_mean(gpu.ctx, 0, None, None, None, None) == ecq.ECQ_ERR_ARG
-    assert L.ecq_decode_mean(gpu.ctx, 65, None, None, None, None) == ecq.ECQ_ERR_ARG
+    assert L.ecq_decode_mean(gpu.ctx, ecq.binding.ECQ_MAX_WORKERS_TOTAL + 1, None, None, None, None) == ecq.ECQ_ERR_ARG
     gpu.close()
 
 
