@@ -19,7 +19,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "ecq_oracle.cpp")
+_SRCS = [os.path.join(_HERE, "ecq_oracle.cpp"), os.path.join(_HERE, "ecq_entropy_oracle.cpp")]
 _LIB = os.path.join(_HERE, "libecq_oracle.so")
 
 STATUS_NONFINITE = 1
@@ -27,12 +27,12 @@ STATUS_NONFINITE = 1
 
 def build(force: bool = False) -> str:
     """Compile the oracle (no optimisation that changes fp32 results)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or \
+            os.path.getmtime(_LIB) < max(os.path.getmtime(p) for p in _SRCS):
         tmp = _LIB + ".tmp.%d" % os.getpid()
         subprocess.check_call([
             "g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math",
-            "-shared", "-fPIC", "-o", tmp, _SRC,
-        ])
+            "-shared", "-fPIC", "-o", tmp] + _SRCS)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -72,6 +72,16 @@ def _load():
         lib.ecqo_entropy_bound_bits.restype = ctypes.c_double
         lib.ecqo_unpack_levels.argtypes = [u64, u32, vp, vp]
         lib.ecqo_unpack_levels.restype = None
+        lib.ecqo_huffman_lengths.argtypes = [vp, u32, u32, vp]
+        lib.ecqo_huffman_lengths.restype = i32
+        lib.ecqo_huffman_words.argtypes = [vp, u32, vp]
+        lib.ecqo_huffman_words.restype = i32
+        lib.ecqo_huffman_chunks.argtypes = [u64]
+        lib.ecqo_huffman_chunks.restype = u64
+        lib.ecqo_huffman_encode.argtypes = [u64, u32, vp, u32, vp, vp, u64, vp]
+        lib.ecqo_huffman_encode.restype = i32
+        lib.ecqo_huffman_decode.argtypes = [u64, u32, vp, u32, vp, vp, vp]
+        lib.ecqo_huffman_decode.restype = i32
         _lib = lib
     return _lib
 
@@ -192,3 +202,63 @@ def unpack_levels(codes: np.ndarray, *, n: int, s: int) -> np.ndarray:
     q = np.zeros(n, dtype=np.int32)
     _load().ecqo_unpack_levels(n, s, _ptr(c), _ptr(q))
     return q
+
+
+# ---- entropy-coded message (paragraph after Eq. 9: "e.g. Huffman") ----------
+HUFFMAN_CHUNK = 1024
+
+
+def huffman_lengths(counts: np.ndarray, *, max_len: int = 12) -> np.ndarray:
+    """Word lengths of an optimal prefix code limited to ``max_len`` bits (0 = absent)."""
+    c = np.ascontiguousarray(counts, dtype=np.uint64)
+    out = np.zeros(c.size, dtype=np.uint8)
+    rc = _load().ecqo_huffman_lengths(_ptr(c), c.size, max_len, _ptr(out))
+    if rc != 0:
+        raise ValueError("alphabet does not fit the length limit")
+    return out
+
+
+def huffman_words(lengths: np.ndarray) -> np.ndarray:
+    """Canonical code words for the given lengths."""
+    L = np.ascontiguousarray(lengths, dtype=np.uint8)
+    out = np.zeros(L.size, dtype=np.uint32)
+    if _load().ecqo_huffman_words(_ptr(L), L.size, _ptr(out)) != 0:
+        raise ValueError("lengths are not those of a prefix code")
+    return out
+
+
+def huffman_chunks(n: int) -> int:
+    return int(_load().ecqo_huffman_chunks(n))
+
+
+def huffman_encode(codes: np.ndarray, lengths: np.ndarray, *, n: int, s: int,
+                   capacity: Optional[int] = None):
+    """Entropy-code one message.  Returns (stream words, chunk offsets)."""
+    r = code_bits(s)
+    c = np.ascontiguousarray(codes, dtype=np.uint32)
+    L = np.ascontiguousarray(lengths, dtype=np.uint8)
+    n_chunks = huffman_chunks(n)
+    cap = capacity if capacity is not None else (n * 32 + 31) // 32 + n_chunks
+    stream = np.zeros(max(cap, 1), dtype=np.uint32)
+    offsets = np.zeros(n_chunks + 1, dtype=np.uint32)
+    rc = _load().ecqo_huffman_encode(n, r, _ptr(L), L.size, _ptr(c), _ptr(stream), cap, _ptr(offsets))
+    if rc == 2:
+        raise OverflowError("stream does not fit the capacity")
+    if rc != 0:
+        raise ValueError("lengths do not cover the message")
+    return stream[:int(offsets[-1])].copy(), offsets
+
+
+def huffman_decode(stream: np.ndarray, offsets: np.ndarray, lengths: np.ndarray, *, n: int,
+                   s: int) -> np.ndarray:
+    """Inverse of :func:`huffman_encode`: the r-bit code words of the message."""
+    r = code_bits(s)
+    st = np.ascontiguousarray(stream, dtype=np.uint32)
+    if st.size == 0:
+        st = np.zeros(1, dtype=np.uint32)
+    off = np.ascontiguousarray(offsets, dtype=np.uint32)
+    L = np.ascontiguousarray(lengths, dtype=np.uint8)
+    out = np.zeros(codes_words(n, s), dtype=np.uint32)
+    if _load().ecqo_huffman_decode(n, r, _ptr(L), L.size, _ptr(st), _ptr(off), _ptr(out)) != 0:
+        raise ValueError("stream holds a bit pattern that is no code word")
+    return out

@@ -11,7 +11,11 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
-# (what is planted, text to replace, replacement)
+ENTROPY = "ecq_entropy_oracle.cpp"
+SOURCES = ("ecq_oracle.cpp", ENTROPY)
+PINS = {"ecq_oracle.cpp": "test_oracle_pins.py", ENTROPY: "test_oracle_entropy.py"}
+
+# (what is planted, text to replace, replacement[, source file])
 MUTATIONS = [
     ("compensation dropped (Eq. 7)", "v[i - lo] = std::fmaf(alpha, h[i], g[i]);", "v[i - lo] = g[i];"),
     ("compensation sign (Eq. 7)", "v[i - lo] = std::fmaf(alpha, h[i], g[i]);", "v[i - lo] = std::fmaf(-alpha, h[i], g[i]);"),
@@ -38,28 +42,41 @@ MUTATIONS = [
      "for (uint64_t j = (hi < i + 32 ? hi : i + 32); j-- > i;) acc = std::fmaf(v[j - lo], v[j - lo], acc);"),
     ("entropy bound in nats", "bits += (double)counts[k] * std::log2(d / (double)counts[k]);", "bits += (double)counts[k] * std::log(d / (double)counts[k]);"),
     ("zero bucket forgets the decay", "const float e = (mode == 0) ? g[i] : vi;\n                h[i] = std::fmaf(beta, h[i], e);", "const float e = (mode == 0) ? g[i] : vi;\n                h[i] = h[i] + e;"),
+    ("package-merge takes one node too many", "for (size_t i = 0; i < 2 * n - 2; ++i) count_leaves", "for (size_t i = 0; i < 2 * n - 1; ++i) count_leaves", ENTROPY),
+    ("package-merge merges without the leaves", "const std::vector<int32_t> leaves = new_leaves();", "const std::vector<int32_t> leaves;", ENTROPY),
+    ("package-merge builds one level too few", "for (uint32_t level = 1; level < max_len; ++level) {", "for (uint32_t level = 2; level < max_len; ++level) {", ENTROPY),
+    ("package-merge builds one level too many", "for (uint32_t level = 1; level < max_len; ++level) {", "for (uint32_t level = 0; level < max_len; ++level) {", ENTROPY),
+    ("packages overlap", "for (size_t i = 0; i + 1 < list.size(); i += 2) {", "for (size_t i = 0; i + 1 < list.size(); i += 1) {", ENTROPY),
+    ("canonical step adds after the shift", "if (i > 0) next = (next + 1) << (L - prev_len);", "if (i > 0) next = (next << (L - prev_len)) + 1;", ENTROPY),
+    ("word sent last bit first", "const uint32_t b = (word[sym] >> (L - 1 - k)) & 1u;", "const uint32_t b = (word[sym] >> k) & 1u;", ENTROPY),
+    ("chunks not aligned to words", "at = (bit + 31) / 32;\n    }\n    if (at > 0xFFFFFFFFull)", "at = bit / 32;\n    }\n    if (at > 0xFFFFFFFFull)", ENTROPY),
+    ("chunk of 1000 entries", "const uint32_t kChunk = 1024;", "const uint32_t kChunk = 1000;", ENTROPY),
+    ("decoder reads the stream from bit 1", "uint64_t bit = (uint64_t)offsets[c] * 32;\n        for (uint64_t i = lo; i < hi; ++i) {\n            uint32_t acc", "uint64_t bit = (uint64_t)offsets[c] * 32 + 1;\n        for (uint64_t i = lo; i < hi; ++i) {\n            uint32_t acc", ENTROPY),
 ]
 
 
-def _run_pins(oracle_dir):
+def _run_pins(oracle_dir, pins):
     env = dict(os.environ)
     env["PYTHONPATH"] = os.path.dirname(oracle_dir) + os.pathsep + ROOT
-    return subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                           os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+    return subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] +
+                          [os.path.join(ROOT, "tests", p) for p in pins],
                           env=env, cwd=os.path.dirname(oracle_dir), capture_output=True, text=True,
                           timeout=900)
 
 
 def test_every_planted_mistake_fails_a_pin(tmp_path):
-    src = open(os.path.join(ROOT, "oracle", "ecq_oracle.cpp")).read()
+    srcs = {f: open(os.path.join(ROOT, "oracle", f)).read() for f in SOURCES}
     def attempt(item):
-        k, (what, old, new) = item
-        assert src.count(old) == 1, "mutation target not found exactly once: " + what
+        k, mutation = item
+        what, old, new = mutation[:3]
+        target = mutation[3] if len(mutation) > 3 else "ecq_oracle.cpp"
+        assert srcs[target].count(old) == 1, "mutation target not found exactly once: " + what
         odir = tmp_path / ("m%02d" % k) / "oracle"
         odir.mkdir(parents=True)
         shutil.copy(os.path.join(ROOT, "oracle", "__init__.py"), odir / "__init__.py")
-        (odir / "ecq_oracle.cpp").write_text(src.replace(old, new))
-        return what if _run_pins(str(odir)).returncode == 0 else None
+        for f in SOURCES:
+            (odir / f).write_text(srcs[f].replace(old, new) if f == target else srcs[f])
+        return what if _run_pins(str(odir), [PINS[target]]).returncode == 0 else None
 
     from concurrent.futures import ThreadPoolExecutor
     with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
@@ -70,7 +87,7 @@ def test_every_planted_mistake_fails_a_pin(tmp_path):
 def test_the_unmutated_copy_passes(tmp_path):
     odir = tmp_path / "clean" / "oracle"
     odir.mkdir(parents=True)
-    for f in ("__init__.py", "ecq_oracle.cpp"):
+    for f in ("__init__.py",) + SOURCES:
         shutil.copy(os.path.join(ROOT, "oracle", f), odir / f)
-    res = _run_pins(str(odir))
+    res = _run_pins(str(odir), list(PINS.values()))
     assert res.returncode == 0, res.stdout[-2000:]
