@@ -161,6 +161,44 @@ def cpu_oracle_sample(w: wl.Workload, sample_elems: int, sample_workers: int):
             "elements_per_s": Ws * n / dt}, dt
 
 
+def entropy_coded_message(ctx, codes, counts_host, w):
+    """Huffman-code one worker's message with the library's coder (outside the timed step):
+    message size and the time of the coder's launches."""
+    import paper_1806_08054_b200 as ecq
+    lengths = ecq.ecq_huffman_lengths(ctx, counts_host)
+    cap = ecq.ecq_huffman_stream_bound(ctx, counts_host, lengths)
+    n_chunks = ecq.ecq_huffman_chunks(ctx)
+    tables = torch.zeros(ecq.ECQ_HUFFMAN_TABLE_BYTES, dtype=torch.uint8, device="cuda")
+    stream = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    offsets = torch.zeros(n_chunks + 1, dtype=torch.int32, device="cuda")
+    back = torch.zeros_like(codes)
+    ecq.ecq_huffman_tables(ctx, lengths, tables)
+
+    def timed(fn, reps=5):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    enc_ms = timed(lambda: ecq.ecq_huffman_encode(ctx, tables, codes, stream, offsets))
+    dec_ms = timed(lambda: ecq.ecq_huffman_decode(ctx, tables, stream, offsets, back))
+    if not torch.equal(back, codes):
+        raise SystemExit("entropy-coded message does not decode to the codes")
+    words = int(offsets[-1].item()) & 0xFFFFFFFF
+    nb = -(-w.d // w.bucket)
+    bits = 32.0 * words + 32.0 * (n_chunks + 1) + 4.0 * len(lengths) + 32.0 * nb
+    return {"bits_per_entry": bits / w.d, "compression": 32.0 * w.d / bits,
+            "payload_bits_per_entry": sum(c * l for c, l in zip(counts_host, lengths)) / w.d,
+            "encode_ms": enc_ms, "decode_ms": dec_ms,
+            "encode_entries_per_s": w.d / (enc_ms * 1e-3), "decode_entries_per_s": w.d / (dec_ms * 1e-3),
+            "includes": "stream, chunk offsets, 4-bit code lengths, fp32 scales"}
+
+
 def run_reference(args, w):
     rank, _, world = dist_env()
     if rank != 0:
@@ -286,7 +324,9 @@ def main():
     # level statistics of worker 0's last message (outside the timed region)
     counts = torch.zeros(2 * w.s + 1, dtype=torch.int64, device="cuda")
     ecq.ecq_code_histogram(ctx, codes[0], counts)
-    entropy_bits = ecq.ecq_entropy_bound_bits(counts.cpu().tolist())
+    counts_host = counts.cpu().tolist()
+    entropy_bits = ecq.ecq_entropy_bound_bits(counts_host)
+    huffman = entropy_coded_message(ctx, codes[0], counts_host, w) if w.s <= 2047 else None
     status = ecq.ecq_status(ctx)
     if status != ecq.ECQ_OK:
         raise SystemExit("codec status %d: %s" % (status, ecq.binding.strerror(status)))
@@ -357,6 +397,7 @@ def main():
                         "compression_fixed": 32.0 / (r + 32.0 / w.bucket),
                         "entropy_bound_bits_per_entry": (entropy_bits + 32.0 * nb) / d,
                         "compression_entropy_bound": 32.0 * d / (entropy_bits + 32.0 * nb),
+                        "huffman": huffman,
                         "note": "worker 0, last timed step; the paper's Table 1 ratios are "
                                 "entropy-coded on other workloads (context only)"},
             # the decode kernel's own bound: one logic instruction per code on the ALU pipe

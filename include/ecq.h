@@ -52,7 +52,9 @@ enum {
     ECQ_ERR_NONFINITE = 3,  /* NaN or Inf met in a compensated gradient (sticky, device) */
     ECQ_ERR_TIMEOUT = 4,    /* a bounded in-kernel wait on an async copy ran out (sticky, device) */
     ECQ_ERR_ALLOC = 5,      /* host or device allocation failed in ecq_create */
-    ECQ_ERR_TOO_LARGE = 6   /* ecq_step_static: the messages do not fit the built-in scratch */
+    ECQ_ERR_TOO_LARGE = 6,  /* ecq_step_static: the messages do not fit the built-in scratch */
+    ECQ_ERR_CAPACITY = 7,   /* ecq_huffman_encode: the stream does not fit the buffer (sticky, device) */
+    ECQ_ERR_SYMBOL = 8      /* a level without a code word / a bit pattern that is no word (sticky, device) */
 };
 
 /*
@@ -187,6 +189,59 @@ int ecq_code_histogram(ecq_ctx* ctx, const uint32_t* codes, uint64_t* counts, vo
 
 /* sum_k d_k log2(d / d_k) over the non-empty bins of HOST counts, d = sum_k d_k. */
 double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins);
+
+/*
+ * Entropy-coded message.  The paragraph after Eq. 9 notes that the r-bit codes can be
+ * compressed further by an entropy code ("e.g. Huffman") with at most
+ * sum_k d_k log2(d / d_k) bits, and the linear-model experiments count their
+ * communication that way.  The paper fixes no format; this one is the library's:
+ *   - a prefix code over the 2s+1 level indices, optimal among codes whose words have at
+ *     most ECQ_HUFFMAN_MAX_LEN bits (Huffman's code whenever that has no longer word);
+ *   - canonical words: symbols ordered by (length, index), the first word all zeros, each
+ *     next one = (previous + 1) shifted left by the growth in length;
+ *   - a word's bits are sent first-bit first into a stream of 32-bit words, bit k of the
+ *     stream being bit k mod 32 of word k / 32;
+ *   - entries are cut into chunks of ECQ_HUFFMAN_CHUNK; every chunk starts on a word
+ *     boundary; offsets[c] is the first word of chunk c, offsets[n_chunks] the stream
+ *     length in words.  A message on the wire is (lengths, offsets, stream, scales).
+ * Available for levels <= 2047 (r <= 12); ECQ_ERR_ARG beyond.
+ *
+ * ecq_huffman_lengths   HOST only: lengths_host[k] (k < 2s+1) from the level counts of
+ *                       ecq_code_histogram, 0 for a level that does not occur, 1 when a
+ *                       single level occurs.
+ * ecq_huffman_chunks    ceil(d / ECQ_HUFFMAN_CHUNK).
+ * ecq_huffman_stream_bound   HOST only: words that are always enough for the stream of a
+ *                       message with these counts under these lengths.
+ * ecq_huffman_tables    builds the encoder and decoder tables of a code from its lengths
+ *                       (HOST, ECQ_ERR_ARG if they are no prefix code) and copies them to
+ *                       tables_dev (ECQ_HUFFMAN_TABLE_BYTES, 16-byte aligned, device) on
+ *                       the stream; lengths_host may be reused when the call returns.
+ * ecq_huffman_encode    codes [ecq_codes_words()] -> stream_words [capacity_words] and
+ *                       offsets [ecq_huffman_chunks() + 1], all device.  If the stream
+ *                       needs more than capacity_words nothing is written to stream_words
+ *                       and ECQ_ERR_CAPACITY becomes pending; a level without a word makes
+ *                       ECQ_ERR_SYMBOL pending (both are read by ecq_status).
+ * ecq_huffman_decode    the inverse: stream_words [stream_len_words], offsets -> codes
+ *                       [ecq_codes_words()], bit-identical to what was encoded.  Nothing
+ *                       beyond stream_len_words is read, whatever the offsets say.  A bit
+ *                       pattern that is no word ends its chunk (rest zero) and makes
+ *                       ECQ_ERR_SYMBOL pending.
+ */
+#define ECQ_HUFFMAN_MAX_LEN 12
+#define ECQ_HUFFMAN_CHUNK 1024
+#define ECQ_HUFFMAN_TABLE_BYTES (4096 * 4 + 4096 * 2)
+int ecq_huffman_lengths(const ecq_ctx* ctx, const uint64_t* counts_host, uint8_t* lengths_host);
+uint64_t ecq_huffman_chunks(const ecq_ctx* ctx);
+uint64_t ecq_huffman_stream_bound(const ecq_ctx* ctx, const uint64_t* counts_host,
+                                  const uint8_t* lengths_host);
+int ecq_huffman_tables(ecq_ctx* ctx, const uint8_t* lengths_host, void* tables_dev,
+                       void* cuda_stream);
+int ecq_huffman_encode(ecq_ctx* ctx, const void* tables_dev, const uint32_t* codes,
+                       uint32_t* stream_words, uint64_t capacity_words, uint32_t* offsets,
+                       void* cuda_stream);
+int ecq_huffman_decode(ecq_ctx* ctx, const void* tables_dev, const uint32_t* stream_words,
+                       uint64_t stream_len_words, const uint32_t* offsets, uint32_t* codes,
+                       void* cuda_stream);
 
 /*
  * One whole iteration from HOST gradients to a HOST result: for every worker

@@ -11,4 +11,6 @@ from .binding import (  # noqa: F401
     ecq_launch_count,
     ecq_num_buckets, ecq_set_error_mode, ecq_set_norm, ecq_status, ecq_step_host, ecq_step_static,
     ecq_step_host_workspace_bytes,
+    ECQ_ERR_CAPACITY, ECQ_ERR_SYMBOL, ECQ_HUFFMAN_TABLE_BYTES, ecq_huffman_chunks, ecq_huffman_decode,
+    ecq_huffman_encode, ecq_huffman_lengths, ecq_huffman_stream_bound, ecq_huffman_tables,
 )

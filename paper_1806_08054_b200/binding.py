@@ -17,6 +17,11 @@ from .build import LIB
 
 ECQ_OK, ECQ_ERR_ARG, ECQ_ERR_CUDA, ECQ_ERR_NONFINITE, ECQ_ERR_TIMEOUT, ECQ_ERR_ALLOC = range(6)
 ECQ_ERR_TOO_LARGE = 6
+ECQ_ERR_CAPACITY = 7
+ECQ_ERR_SYMBOL = 8
+ECQ_HUFFMAN_MAX_LEN = 12
+ECQ_HUFFMAN_CHUNK = 1024
+ECQ_HUFFMAN_TABLE_BYTES = 4096 * 4 + 4096 * 2
 ECQ_STATIC_SCRATCH_BYTES = 4 << 20
 ECQ_MAX_WORKERS = 64
 ECQ_MAX_WORKERS_TOTAL = 1024
@@ -73,6 +78,18 @@ def lib() -> ctypes.CDLL:
         L.ecq_step_host.restype = i32
         L.ecq_step_static.argtypes = [u64, u32, u32, f32, f32, u64, u32, u32, vp, vp, vp, vp]
         L.ecq_step_static.restype = i32
+        L.ecq_huffman_lengths.argtypes = [vp, vp, vp]
+        L.ecq_huffman_lengths.restype = i32
+        L.ecq_huffman_chunks.argtypes = [vp]
+        L.ecq_huffman_chunks.restype = u64
+        L.ecq_huffman_stream_bound.argtypes = [vp, vp, vp]
+        L.ecq_huffman_stream_bound.restype = u64
+        L.ecq_huffman_tables.argtypes = [vp, vp, vp, vp]
+        L.ecq_huffman_tables.restype = i32
+        L.ecq_huffman_encode.argtypes = [vp, vp, vp, vp, u64, vp, vp]
+        L.ecq_huffman_encode.restype = i32
+        L.ecq_huffman_decode.argtypes = [vp, vp, vp, u64, vp, vp, vp]
+        L.ecq_huffman_decode.restype = i32
         L.ecq_status.argtypes = [vp, vp]
         L.ecq_status.restype = i32
         L.ecq_launch_count.argtypes = []
@@ -251,3 +268,65 @@ def ecq_status(ctx: int, stream=None) -> int:
 
 def ecq_launch_count() -> int:
     return int(lib().ecq_launch_count())
+
+
+# ---- entropy-coded message ----------------------------------------------------
+def _host_u64(counts, n):
+    arr = (ctypes.c_uint64 * n)(*[int(x) for x in counts])
+    return arr
+
+
+def ecq_huffman_lengths(ctx: int, counts) -> list:
+    """Code-word lengths (host list of 2s+1 ints) from the level counts of a message."""
+    n = len(counts)
+    c = _host_u64(counts, n)
+    out = (ctypes.c_uint8 * n)()
+    rc = lib().ecq_huffman_lengths(ctx, c, out)
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_huffman_lengths")
+    return list(out)
+
+
+def ecq_huffman_chunks(ctx: int) -> int:
+    return int(lib().ecq_huffman_chunks(ctx))
+
+
+def ecq_huffman_stream_bound(ctx: int, counts, lengths) -> int:
+    """Stream words that always suffice for a message with these counts and lengths."""
+    n = len(counts)
+    return int(lib().ecq_huffman_stream_bound(ctx, _host_u64(counts, n),
+                                               (ctypes.c_uint8 * n)(*[int(x) for x in lengths])))
+
+
+def ecq_huffman_tables(ctx: int, lengths, tables: torch.Tensor, stream=None) -> None:
+    """Build the tables of the code with these lengths into ``tables`` (uint8 CUDA tensor
+    of ECQ_HUFFMAN_TABLE_BYTES)."""
+    if tables.numel() < ECQ_HUFFMAN_TABLE_BYTES:
+        raise ValueError("tables must hold ECQ_HUFFMAN_TABLE_BYTES bytes")
+    n = len(lengths)
+    rc = lib().ecq_huffman_tables(ctx, (ctypes.c_uint8 * n)(*[int(x) for x in lengths]),
+                                  _dev(tables, torch.uint8, "tables"), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_huffman_tables")
+
+
+def ecq_huffman_encode(ctx: int, tables: torch.Tensor, codes: torch.Tensor, stream_words: torch.Tensor,
+                       offsets: torch.Tensor, stream=None) -> None:
+    """Enqueue the entropy coder: ``codes`` -> ``stream_words`` (its size is the capacity)
+    and ``offsets`` (ecq_huffman_chunks() + 1 words)."""
+    rc = lib().ecq_huffman_encode(ctx, _dev(tables, torch.uint8, "tables"), _dev(codes, torch.int32, "codes"),
+                                  _dev(stream_words, torch.int32, "stream_words"), stream_words.numel(),
+                                  _dev(offsets, torch.int32, "offsets"), _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_huffman_encode")
+
+
+def ecq_huffman_decode(ctx: int, tables: torch.Tensor, stream_words: torch.Tensor, offsets: torch.Tensor,
+                       codes: torch.Tensor, stream=None) -> None:
+    """Enqueue the inverse of :func:`ecq_huffman_encode`."""
+    rc = lib().ecq_huffman_decode(ctx, _dev(tables, torch.uint8, "tables"),
+                                  _dev(stream_words, torch.int32, "stream_words"), stream_words.numel(),
+                                  _dev(offsets, torch.int32, "offsets"), _dev(codes, torch.int32, "codes"),
+                                  _stream(stream))
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_huffman_decode")

@@ -7,6 +7,8 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
+#include <vector>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -16,6 +18,7 @@
 #include "ecq_decode.cuh"
 #include "ecq_encode.cuh"
 #include "ecq_stats.cuh"
+#include "ecq_entropy.cuh"
 
 using namespace ecq;
 
@@ -457,6 +460,145 @@ double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins) {
     return bits;
 }
 
+// ---- entropy-coded message ---------------------------------------------------------------
+// Length-limited Huffman lengths by package-merge, kept as sorted weight lists: level L
+// (the deepest) holds the leaves; the list of a level is the merge of the leaves with the
+// pairs of the level below.  Only how many of a list's first k entries are leaves is
+// needed to read the lengths off: the k_1 = 2n - 2 cheapest entries of the top list
+// contain a_1 leaves and k_1 - a_1 packages, which are the first 2 (k_1 - a_1) entries of
+// the next list, and so on; the i-th lightest symbol gets one bit per level with a_j > i.
+int ecq_huffman_lengths(const ecq_ctx* c, const uint64_t* counts_host, uint8_t* lengths_host) {
+    if (!c || !counts_host || !lengths_host) return ECQ_ERR_ARG;
+    const uint32_t n_sym = 2 * c->P.s + 1;
+    if (n_sym > kHuffMaxSymbols) return ECQ_ERR_ARG;
+    std::vector<std::pair<uint64_t, uint32_t>> leaf;          // (count, symbol), ascending
+    for (uint32_t k = 0; k < n_sym; ++k) {
+        lengths_host[k] = 0;
+        if (counts_host[k]) leaf.emplace_back(counts_host[k], k);
+    }
+    const size_t n = leaf.size();
+    if (n == 0) return ECQ_OK;
+    if (n == 1) { lengths_host[leaf[0].second] = 1; return ECQ_OK; }
+    std::sort(leaf.begin(), leaf.end());
+    struct Level { std::vector<uint64_t> weight; std::vector<uint8_t> is_leaf; };
+    std::vector<Level> level(kHuffMaxLen);                   // [0] top ... [L-1] deepest
+    Level& deepest = level[kHuffMaxLen - 1];
+    for (size_t i = 0; i < n; ++i) { deepest.weight.push_back(leaf[i].first); deepest.is_leaf.push_back(1); }
+    for (int j = (int)kHuffMaxLen - 2; j >= 0; --j) {
+        const Level& below = level[j + 1];
+        Level& here = level[j];
+        size_t a = 0, b = 0;
+        const size_t n_pairs = below.weight.size() / 2;
+        while (a < n || b < n_pairs) {
+            const uint64_t pw = b < n_pairs ? below.weight[2 * b] + below.weight[2 * b + 1] : 0;
+            if (b == n_pairs || (a < n && leaf[a].first <= pw)) {
+                here.weight.push_back(leaf[a].first); here.is_leaf.push_back(1); ++a;
+            } else {
+                here.weight.push_back(pw); here.is_leaf.push_back(0); ++b;
+            }
+        }
+    }
+    size_t take = 2 * n - 2;
+    for (uint32_t j = 0; j < kHuffMaxLen && take > 0; ++j) {
+        size_t leaves = 0;
+        for (size_t i = 0; i < take; ++i) leaves += level[j].is_leaf[i];
+        for (size_t i = 0; i < leaves; ++i) lengths_host[leaf[i].second] += 1;
+        take = 2 * (take - leaves);
+    }
+    return ECQ_OK;
+}
+
+uint64_t ecq_huffman_chunks(const ecq_ctx* c) {
+    return c ? (c->P.d + kHuffChunk - 1) / kHuffChunk : 0;
+}
+
+uint64_t ecq_huffman_stream_bound(const ecq_ctx* c, const uint64_t* counts_host,
+                                  const uint8_t* lengths_host) {
+    if (!c || !counts_host || !lengths_host) return 0;
+    const uint32_t n_sym = 2 * c->P.s + 1;
+    uint64_t bits = 0;
+    for (uint32_t k = 0; k < n_sym; ++k) bits += counts_host[k] * lengths_host[k];
+    return (bits + 31) / 32 + ecq_huffman_chunks(c);
+}
+
+int ecq_huffman_tables(ecq_ctx* c, const uint8_t* lengths_host, void* tables_dev, void* cuda_stream) {
+    if (!c || !lengths_host || !tables_dev || !aligned16(tables_dev)) return ECQ_ERR_ARG;
+    const uint32_t n_sym = 2 * c->P.s + 1;
+    if (n_sym > kHuffMaxSymbols) return ECQ_ERR_ARG;
+    // canonical words: within a length in symbol order, the first word of a length is the
+    // first unused word of the previous length with a zero appended
+    uint32_t per_len[kHuffMaxLen + 2] = {0}, first[kHuffMaxLen + 2] = {0};
+    uint64_t kraft = 0;
+    for (uint32_t k = 0; k < n_sym; ++k) {
+        if (lengths_host[k] > kHuffMaxLen) return ECQ_ERR_ARG;
+        if (lengths_host[k]) { per_len[lengths_host[k]] += 1; kraft += 1ull << (kHuffMaxLen - lengths_host[k]); }
+    }
+    if (kraft > (1ull << kHuffMaxLen)) return ECQ_ERR_ARG;
+    for (uint32_t L = 1; L <= kHuffMaxLen; ++L) first[L] = (first[L - 1] + per_len[L - 1]) << 1;
+    HuffTables* t = new (std::nothrow) HuffTables;
+    if (!t) return ECQ_ERR_ALLOC;
+    std::memset(t, 0, sizeof(*t));
+    for (uint32_t k = 0; k < n_sym; ++k) {
+        const uint32_t L = lengths_host[k];
+        if (!L) continue;
+        const uint32_t word = first[L]++;
+        uint32_t rev = 0;                                    // first bit sent -> bit 0
+        for (uint32_t b = 0; b < L; ++b) rev |= ((word >> (L - 1 - b)) & 1u) << b;
+        t->enc[k] = (L << 16) | rev;
+        for (uint32_t hi = 0; hi < (1u << (kHuffMaxLen - L)); ++hi)
+            t->dec[(hi << L) | rev] = (uint16_t)((k << 4) | L);
+    }
+    // pageable source: the copy is staged before the call returns, so `t` can go
+    const cudaError_t e = cudaMemcpyAsync(tables_dev, t, sizeof(*t), cudaMemcpyHostToDevice,
+                                          static_cast<cudaStream_t>(cuda_stream));
+    delete t;
+    return e == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+int ecq_huffman_encode(ecq_ctx* c, const void* tables_dev, const uint32_t* codes,
+                       uint32_t* stream_words, uint64_t capacity_words, uint32_t* offsets,
+                       void* cuda_stream) {
+    if (!c || !tables_dev || !codes || !stream_words || !offsets || !aligned16(tables_dev) ||
+        !aligned16(codes) || !aligned4(stream_words) || !aligned4(offsets))
+        return ECQ_ERR_ARG;
+    const uint32_t n_sym = 2 * c->P.s + 1;
+    if (n_sym > kHuffMaxSymbols) return ECQ_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const HuffTables* t = static_cast<const HuffTables*>(tables_dev);
+    const uint64_t n_chunks = ecq_huffman_chunks(c);
+    uint64_t blocks = (n_chunks + kHuffWarps - 1) / kHuffWarps;
+    const uint64_t cap = (uint64_t)c->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    const size_t smem_count = (size_t)n_sym * 4;
+    const size_t smem_write = ((size_t)((n_sym + 31) & ~31u) + kHuffWarps * (kHuffChunkWords + 32)) * 4;
+    huff_count_kernel<<<(uint32_t)blocks, kHuffWarps * 32, smem_count, st>>>(
+        c->P, t, codes, offsets, c->d_status, n_chunks);
+    huff_scan_kernel<<<1, kScanThreads, 0, st>>>(offsets, n_chunks, capacity_words, c->d_status);
+    huff_write_kernel<<<(uint32_t)blocks, kHuffWarps * 32, smem_write, st>>>(
+        c->P, t, codes, offsets, stream_words, n_chunks);
+    g_launches.fetch_add(3, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
+int ecq_huffman_decode(ecq_ctx* c, const void* tables_dev, const uint32_t* stream_words,
+                       uint64_t stream_len_words, const uint32_t* offsets, uint32_t* codes,
+                       void* cuda_stream) {
+    if (!c || !tables_dev || !stream_words || !offsets || !codes || !aligned16(tables_dev) ||
+        !aligned4(stream_words) || !aligned4(offsets) || !aligned16(codes))
+        return ECQ_ERR_ARG;
+    const uint32_t n_sym = 2 * c->P.s + 1;
+    if (n_sym > kHuffMaxSymbols) return ECQ_ERR_ARG;
+    const uint64_t n_chunks = ecq_huffman_chunks(c);
+    uint64_t blocks = (n_chunks + kHuffDecThreads - 1) / kHuffDecThreads;
+    const uint64_t cap = (uint64_t)c->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    huff_decode_kernel<<<(uint32_t)blocks, kHuffDecThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        c->P, static_cast<const HuffTables*>(tables_dev), stream_words, offsets, codes, c->d_status,
+        n_chunks, c->n_words, stream_len_words);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
+}
+
 uint64_t ecq_step_host_workspace_bytes(const ecq_ctx* c, uint32_t W) {
     if (!c || W == 0 || W > ECQ_MAX_WORKERS) return 0;
     const uint64_t stage = round_up(c->P.d * 4, 256);
@@ -536,6 +678,8 @@ int ecq_status(ecq_ctx* c, void* cuda_stream) {
     const uint32_t bits = *c->h_status;
     if (bits & kStatusTimeout) return ECQ_ERR_TIMEOUT;
     if (bits & kStatusNonFinite) return ECQ_ERR_NONFINITE;
+    if (bits & kStatusCapacity) return ECQ_ERR_CAPACITY;
+    if (bits & kStatusSymbol) return ECQ_ERR_SYMBOL;
     return ECQ_OK;
 }
 
@@ -550,6 +694,8 @@ const char* ecq_strerror(int status) {
         case ECQ_ERR_TIMEOUT: return "an in-kernel wait on an asynchronous copy ran out";
         case ECQ_ERR_ALLOC: return "allocation failed";
         case ECQ_ERR_TOO_LARGE: return "problem too large for the built-in scratch of ecq_step_static";
+        case ECQ_ERR_CAPACITY: return "the entropy-coded stream does not fit the given buffer";
+        case ECQ_ERR_SYMBOL: return "a level without a code word, or a bit pattern that is no code word";
         default: return "unknown status";
     }
 }
@@ -651,5 +797,7 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
     if (rc != ECQ_OK) return rc;
     if (bits & kStatusTimeout) return ECQ_ERR_TIMEOUT;
     if (bits & kStatusNonFinite) return ECQ_ERR_NONFINITE;
+    if (bits & kStatusCapacity) return ECQ_ERR_CAPACITY;
+    if (bits & kStatusSymbol) return ECQ_ERR_SYMBOL;
     return ECQ_OK;
 }
