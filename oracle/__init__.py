@@ -78,9 +78,9 @@ def _load():
         lib.ecqo_huffman_words.restype = i32
         lib.ecqo_huffman_chunks.argtypes = [u64]
         lib.ecqo_huffman_chunks.restype = u64
-        lib.ecqo_huffman_encode.argtypes = [u64, u32, vp, u32, vp, vp, u64, vp]
+        lib.ecqo_huffman_encode.argtypes = [u64, u32, vp, u32, vp, vp, u64, vp, vp]
         lib.ecqo_huffman_encode.restype = i32
-        lib.ecqo_huffman_decode.argtypes = [u64, u32, vp, u32, vp, vp, vp]
+        lib.ecqo_huffman_decode.argtypes = [u64, u32, vp, u32, vp, vp, vp, vp]
         lib.ecqo_huffman_decode.restype = i32
         _lib = lib
     return _lib
@@ -233,7 +233,7 @@ def huffman_chunks(n: int) -> int:
 
 def huffman_encode(codes: np.ndarray, lengths: np.ndarray, *, n: int, s: int,
                    capacity: Optional[int] = None):
-    """Entropy-code one message.  Returns (stream words, chunk offsets)."""
+    """Entropy-code one message.  Returns (stream words, chunk offsets, quarter positions)."""
     r = code_bits(s)
     c = np.ascontiguousarray(codes, dtype=np.uint32)
     L = np.ascontiguousarray(lengths, dtype=np.uint8)
@@ -241,24 +241,29 @@ def huffman_encode(codes: np.ndarray, lengths: np.ndarray, *, n: int, s: int,
     cap = capacity if capacity is not None else (n * 32 + 31) // 32 + n_chunks
     stream = np.zeros(max(cap, 1), dtype=np.uint32)
     offsets = np.zeros(n_chunks + 1, dtype=np.uint32)
-    rc = _load().ecqo_huffman_encode(n, r, _ptr(L), L.size, _ptr(c), _ptr(stream), cap, _ptr(offsets))
+    quarters = np.zeros(3 * n_chunks, dtype=np.uint16)
+    rc = _load().ecqo_huffman_encode(n, r, _ptr(L), L.size, _ptr(c), _ptr(stream), cap, _ptr(offsets),
+                                     _ptr(quarters))
     if rc == 2:
         raise OverflowError("stream does not fit the capacity")
     if rc != 0:
         raise ValueError("lengths do not cover the message")
-    return stream[:int(offsets[-1])].copy(), offsets
+    return stream[:int(offsets[-1])].copy(), offsets, quarters
 
 
-def huffman_decode(stream: np.ndarray, offsets: np.ndarray, lengths: np.ndarray, *, n: int,
-                   s: int) -> np.ndarray:
+def huffman_decode(stream: np.ndarray, offsets: np.ndarray, quarters: np.ndarray,
+                   lengths: np.ndarray, *, n: int, s: int) -> np.ndarray:
     """Inverse of :func:`huffman_encode`: the r-bit code words of the message."""
     r = code_bits(s)
     st = np.ascontiguousarray(stream, dtype=np.uint32)
     if st.size == 0:
         st = np.zeros(1, dtype=np.uint32)
     off = np.ascontiguousarray(offsets, dtype=np.uint32)
+    qt = np.ascontiguousarray(quarters, dtype=np.uint16)
+    if qt.size == 0:
+        qt = np.zeros(3, dtype=np.uint16)
     L = np.ascontiguousarray(lengths, dtype=np.uint8)
     out = np.zeros(codes_words(n, s), dtype=np.uint32)
-    if _load().ecqo_huffman_decode(n, r, _ptr(L), L.size, _ptr(st), _ptr(off), _ptr(out)) != 0:
+    if _load().ecqo_huffman_decode(n, r, _ptr(L), L.size, _ptr(st), _ptr(off), _ptr(qt), _ptr(out)) != 0:
         raise ValueError("stream holds a bit pattern that is no code word")
     return out

@@ -21,7 +21,11 @@
 //     bit k is bit (k mod 32) of word k / 32;
 //   * the entries are cut into chunks of 1024; every chunk starts on a word
 //     boundary, offsets[c] is its first word and offsets[n_chunks] the length
-//     of the stream in words (unused bits of a chunk's last word are zero).
+//     of the stream in words (unused bits of a chunk's last word are zero);
+//   * so that a chunk can be decoded by four independent readers, quarters[3c + j]
+//     (j = 0, 1, 2) is the bit position, counted from the chunk's first word, at
+//     which entry 256 (j + 1) of the chunk starts (the chunk's end if it has fewer
+//     entries).
 //
 // Pins (tests/test_oracle_entropy.py): exhaustive search over all admissible
 // length vectors on tiny alphabets; a textbook six-symbol example; Huffman's
@@ -36,6 +40,7 @@
 namespace {
 
 const uint32_t kChunk = 1024;
+const uint32_t kQuarter = 256;
 
 uint32_t get_bits(const uint32_t* words, uint64_t bit, uint32_t n) {
     uint32_t v = 0;
@@ -154,11 +159,12 @@ int ecqo_huffman_words(const uint8_t* lengths, uint32_t n_sym, uint32_t* words) 
 uint64_t ecqo_huffman_chunks(uint64_t n) { return (n + kChunk - 1) / kChunk; }
 
 // Entropy-code the n r-bit codes of `codes`.  stream must hold `capacity` words;
-// offsets n_chunks + 1 entries.  Returns 0; 1 for lengths that are no prefix code or
-// a symbol without a word; 2 if the stream does not fit (nothing useful is written).
+// offsets n_chunks + 1 entries, quarters 3 n_chunks.  Returns 0; 1 for lengths that are no
+// prefix code or a symbol without a word; 2 if the stream does not fit (nothing useful is
+// written).
 int ecqo_huffman_encode(uint64_t n, uint32_t r, const uint8_t* lengths, uint32_t n_sym,
                         const uint32_t* codes, uint32_t* stream, uint64_t capacity,
-                        uint32_t* offsets) {
+                        uint32_t* offsets, uint16_t* quarters) {
     std::vector<uint32_t> word;
     if (!canonical_words(lengths, n_sym, word)) return 1;
     const uint64_t n_chunks = ecqo_huffman_chunks(n);
@@ -167,7 +173,10 @@ int ecqo_huffman_encode(uint64_t n, uint32_t r, const uint8_t* lengths, uint32_t
         offsets[c] = (uint32_t)at;
         const uint64_t lo = c * kChunk, hi = std::min<uint64_t>(n, lo + kChunk);
         uint64_t bit = at * 32;
+        for (uint32_t j = 0; j < 3; ++j) quarters[3 * c + j] = 0;
         for (uint64_t i = lo; i < hi; ++i) {
+            if (i > lo && (i - lo) % kQuarter == 0)
+                quarters[3 * c + (i - lo) / kQuarter - 1] = (uint16_t)(bit - at * 32);
             const uint32_t sym = get_bits(codes, i * r, r);
             if (sym >= n_sym || lengths[sym] == 0) return 1;
             const uint32_t L = lengths[sym];
@@ -179,6 +188,8 @@ int ecqo_huffman_encode(uint64_t n, uint32_t r, const uint8_t* lengths, uint32_t
                 ++bit;
             }
         }
+        for (uint64_t q = (hi - lo + kQuarter - 1) / kQuarter; q < 4; ++q)   // quarters that do not exist
+            if (q > 0) quarters[3 * c + q - 1] = (uint16_t)(bit - at * 32);
         at = (bit + 31) / 32;
     }
     if (at > 0xFFFFFFFFull) return 2;
@@ -187,10 +198,12 @@ int ecqo_huffman_encode(uint64_t n, uint32_t r, const uint8_t* lengths, uint32_t
 }
 
 // Inverse: walks the stream bit by bit, extending the current word until it equals a
-// code word of that length.  Writes the n symbols as r-bit codes (unused bits of the
-// last word zero).  Returns 0, or 1 on a bit pattern that is no code word.
+// code word of that length; every quarter of a chunk is entered at its recorded bit
+// position.  Writes the n symbols as r-bit codes (unused bits of the last word zero).
+// Returns 0, or 1 on a bit pattern that is no code word.
 int ecqo_huffman_decode(uint64_t n, uint32_t r, const uint8_t* lengths, uint32_t n_sym,
-                        const uint32_t* stream, const uint32_t* offsets, uint32_t* codes) {
+                        const uint32_t* stream, const uint32_t* offsets,
+                        const uint16_t* quarters, uint32_t* codes) {
     std::vector<uint32_t> word;
     if (!canonical_words(lengths, n_sym, word)) return 1;
     std::vector<std::vector<uint32_t>> of_length(33);      // the symbols of every word length
@@ -203,6 +216,8 @@ int ecqo_huffman_decode(uint64_t n, uint32_t r, const uint8_t* lengths, uint32_t
         const uint64_t lo = c * kChunk, hi = std::min<uint64_t>(n, lo + kChunk);
         uint64_t bit = (uint64_t)offsets[c] * 32;
         for (uint64_t i = lo; i < hi; ++i) {
+            if (i > lo && (i - lo) % kQuarter == 0)
+                bit = (uint64_t)offsets[c] * 32 + quarters[3 * c + (i - lo) / kQuarter - 1];
             uint32_t acc = 0, L = 0, sym = n_sym;
             while (sym == n_sym) {
                 if (L == 32) return 1;

@@ -174,8 +174,9 @@ def test_hand_packed_stream():
     # 0 10 11 0 0 11 10, first bit in bit 0 of the word:
     # bits 1, 3, 4, 7, 8, 9 are set -> 2 + 8 + 16 + 128 + 256 + 512 = 922.
     L = np.array([2, 1, 2], dtype=np.uint8)
-    stream, offsets = oracle.huffman_encode(pack([1, 0, 2, 1, 1, 2, 0], 2), L, n=7, s=1)
+    stream, offsets, quarters = oracle.huffman_encode(pack([1, 0, 2, 1, 1, 2, 0], 2), L, n=7, s=1)
     assert stream.tolist() == [922] and offsets.tolist() == [0, 1]
+    assert quarters.tolist() == [11, 11, 11]          # no entry 256, 512, 768: the chunk's end
 
 
 def test_chunks_start_on_word_boundaries():
@@ -183,13 +184,21 @@ def test_chunks_start_on_word_boundaries():
     # even when the first does not end on a boundary
     L = np.array([2, 1, 2], dtype=np.uint8)
     msg = [1] * 1024 + [2]
-    stream, offsets = oracle.huffman_encode(pack(msg, 2), L, n=1025, s=1)
+    stream, offsets, quarters = oracle.huffman_encode(pack(msg, 2), L, n=1025, s=1)
     assert offsets.tolist() == [0, 32, 33] and stream[:32].tolist() == [0] * 32 and stream[32] == 3
+    # one bit per entry in chunk 0: its quarters start at bits 256, 512, 768; chunk 1 has
+    # one entry of two bits and no further quarter
+    assert quarters.tolist() == [256, 512, 768, 2, 2, 2]
     msg = [1] * 1023 + [0] + [2, 1, 0]
-    stream, offsets = oracle.huffman_encode(pack(msg, 2), L, n=1027, s=1)
+    stream, offsets, quarters = oracle.huffman_encode(pack(msg, 2), L, n=1027, s=1)
     # chunk 0: 1023 zeros then "10" = 1025 bits -> 33 words, bit 1023 set; chunk 1: 11 0 10
     assert offsets.tolist() == [0, 33, 34]
     assert stream[31] == 1 << 31 and stream[32] == 0 and stream[33] == 0b01011
+    assert quarters.tolist() == [256, 512, 768, 5, 5, 5]
+    # two-bit words in the second quarter shift the later marks
+    msg = [1] * 256 + [0] * 256 + [1] * 300
+    _, _, quarters = oracle.huffman_encode(pack(msg, 2), L, n=812, s=1)
+    assert quarters.tolist() == [256, 768, 1024]
 
 
 @pytest.mark.parametrize("s", [1, 2, 4, 8, 128, 300, 2047])
@@ -208,15 +217,29 @@ def test_round_trip_and_length(s):
         counts = oracle.code_histogram(codes, n=n, s=s)
         assert counts.sum() == n and np.array_equal(counts, np.bincount(sym, minlength=2 * s + 1))
         L = oracle.huffman_lengths(counts, max_len=12)
-        stream, offsets = oracle.huffman_encode(codes, L, n=n, s=s)
+        stream, offsets, quarters = oracle.huffman_encode(codes, L, n=n, s=s)
         n_chunks = -(-n // 1024)
+        # a quarter mark is the number of bits the entries before it take
+        for c in range(n_chunks):
+            lens = L[sym[c * 1024:(c + 1) * 1024]].astype(np.int64)
+            cum = np.concatenate([[0], np.cumsum(lens)])
+            want = [int(cum[min(256 * (j + 1), lens.size)]) for j in range(3)]
+            assert quarters[3 * c:3 * c + 3].tolist() == want
         assert offsets.size == n_chunks + 1 and offsets[0] == 0 and offsets[-1] == stream.size
         # every chunk takes exactly the words its symbols need
         for c in range(n_chunks):
             bits_c = int(L[sym[c * 1024:(c + 1) * 1024]].astype(np.int64).sum())
             assert offsets[c + 1] - offsets[c] == -(-bits_c // 32)
-        back = oracle.huffman_decode(stream, offsets, L, n=n, s=s)
+        back = oracle.huffman_decode(stream, offsets, quarters, L, n=n, s=s)
         assert np.array_equal(back, codes)
+        if n > 256 and np.count_nonzero(counts) > 1:
+            # the quarters are really entered at their marks: a wrong mark breaks the decode
+            wrong = quarters.copy()
+            wrong[0] += 1
+            try:
+                assert not np.array_equal(oracle.huffman_decode(stream, offsets, wrong, L, n=n, s=s), codes)
+            except ValueError:
+                pass
         # Huffman: within one bit per symbol of the entropy bound, never below it
         payload = cost(counts, L)
         H = oracle.entropy_bound_bits(counts)

@@ -51,7 +51,9 @@ MUTATIONS = [
     ("word sent last bit first", "const uint32_t b = (word[sym] >> (L - 1 - k)) & 1u;", "const uint32_t b = (word[sym] >> k) & 1u;", ENTROPY),
     ("chunks not aligned to words", "at = (bit + 31) / 32;\n    }\n    if (at > 0xFFFFFFFFull)", "at = bit / 32;\n    }\n    if (at > 0xFFFFFFFFull)", ENTROPY),
     ("chunk of 1000 entries", "const uint32_t kChunk = 1024;", "const uint32_t kChunk = 1000;", ENTROPY),
-    ("decoder reads the stream from bit 1", "uint64_t bit = (uint64_t)offsets[c] * 32;\n        for (uint64_t i = lo; i < hi; ++i) {\n            uint32_t acc", "uint64_t bit = (uint64_t)offsets[c] * 32 + 1;\n        for (uint64_t i = lo; i < hi; ++i) {\n            uint32_t acc", ENTROPY),
+    ("quarter marks one entry late", "if (i > lo && (i - lo) % kQuarter == 0)\n                quarters[3 * c + (i - lo) / kQuarter - 1] = (uint16_t)(bit - at * 32);\n            const uint32_t sym = get_bits(codes, i * r, r);", "const uint32_t sym = get_bits(codes, i * r, r);\n            if (i > lo && (i - lo) % kQuarter == 0)\n                quarters[3 * c + (i - lo) / kQuarter - 1] = (uint16_t)(bit - at * 32 + lengths[sym < n_sym ? sym : 0]);", ENTROPY),
+    ("quarter of 128 entries", "const uint32_t kQuarter = 256;", "const uint32_t kQuarter = 128;", ENTROPY),
+    ("decoder reads the stream from bit 1", "uint64_t bit = (uint64_t)offsets[c] * 32;\n        for (uint64_t i = lo; i < hi; ++i) {\n            if (i > lo && (i - lo) % kQuarter == 0)\n                bit =", "uint64_t bit = (uint64_t)offsets[c] * 32 + 1;\n        for (uint64_t i = lo; i < hi; ++i) {\n            if (i > lo && (i - lo) % kQuarter == 0)\n                bit =", ENTROPY),
 ]
 
 
