@@ -171,6 +171,7 @@ def entropy_coded_message(ctx, codes, counts_host, w):
     tables = torch.zeros(ecq.ECQ_HUFFMAN_TABLE_BYTES, dtype=torch.uint8, device="cuda")
     stream = torch.zeros(cap, dtype=torch.int32, device="cuda")
     offsets = torch.zeros(n_chunks + 1, dtype=torch.int32, device="cuda")
+    quarters = torch.zeros(3 * n_chunks, dtype=torch.int16, device="cuda")
     back = torch.zeros_like(codes)
     ecq.ecq_huffman_tables(ctx, lengths, tables)
 
@@ -185,18 +186,18 @@ def entropy_coded_message(ctx, codes, counts_host, w):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps
 
-    enc_ms = timed(lambda: ecq.ecq_huffman_encode(ctx, tables, codes, stream, offsets))
-    dec_ms = timed(lambda: ecq.ecq_huffman_decode(ctx, tables, stream, offsets, back))
+    enc_ms = timed(lambda: ecq.ecq_huffman_encode(ctx, tables, codes, stream, offsets, quarters))
+    dec_ms = timed(lambda: ecq.ecq_huffman_decode(ctx, tables, stream, offsets, quarters, back))
     if not torch.equal(back, codes):
         raise SystemExit("entropy-coded message does not decode to the codes")
     words = int(offsets[-1].item()) & 0xFFFFFFFF
     nb = -(-w.d // w.bucket)
-    bits = 32.0 * words + 32.0 * (n_chunks + 1) + 4.0 * len(lengths) + 32.0 * nb
+    bits = 32.0 * words + 32.0 * (n_chunks + 1) + 48.0 * n_chunks + 4.0 * len(lengths) + 32.0 * nb
     return {"bits_per_entry": bits / w.d, "compression": 32.0 * w.d / bits,
             "payload_bits_per_entry": sum(c * l for c, l in zip(counts_host, lengths)) / w.d,
             "encode_ms": enc_ms, "decode_ms": dec_ms,
             "encode_entries_per_s": w.d / (enc_ms * 1e-3), "decode_entries_per_s": w.d / (dec_ms * 1e-3),
-            "includes": "stream, chunk offsets, 4-bit code lengths, fp32 scales"}
+            "includes": "stream, chunk offsets, quarter marks, 4-bit code lengths, fp32 scales"}
 
 
 def run_reference(args, w):

@@ -203,7 +203,11 @@ double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins);
  *     stream being bit k mod 32 of word k / 32;
  *   - entries are cut into chunks of ECQ_HUFFMAN_CHUNK; every chunk starts on a word
  *     boundary; offsets[c] is the first word of chunk c, offsets[n_chunks] the stream
- *     length in words.  A message on the wire is (lengths, offsets, stream, scales).
+ *     length in words;
+ *   - quarters[3c + j] (j = 0, 1, 2) is the bit, counted from the first word of chunk c,
+ *     at which entry 256 (j + 1) of that chunk starts (the chunk's end if it has fewer
+ *     entries): four readers can share a chunk.
+ *     A message on the wire is (lengths, offsets, quarters, stream, scales).
  * Available for levels <= 2047 (r <= 12); ECQ_ERR_ARG beyond.
  *
  * ecq_huffman_lengths   HOST only: lengths_host[k] (k < 2s+1) from the level counts of
@@ -216,20 +220,21 @@ double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins);
  *                       (HOST, ECQ_ERR_ARG if they are no prefix code) and copies them to
  *                       tables_dev (ECQ_HUFFMAN_TABLE_BYTES, 16-byte aligned, device) on
  *                       the stream; lengths_host may be reused when the call returns.
- * ecq_huffman_encode    codes [ecq_codes_words()] -> stream_words [capacity_words] and
- *                       offsets [ecq_huffman_chunks() + 1], all device.  If the stream
+ * ecq_huffman_encode    codes [ecq_codes_words()] -> stream_words [capacity_words],
+ *                       offsets [ecq_huffman_chunks() + 1] and quarters
+ *                       [3 * ecq_huffman_chunks()], all device.  If the stream
  *                       needs more than capacity_words nothing is written to stream_words
  *                       and ECQ_ERR_CAPACITY becomes pending; a level without a word makes
  *                       ECQ_ERR_SYMBOL pending (both are read by ecq_status).
- * ecq_huffman_decode    the inverse: stream_words [stream_len_words], offsets -> codes
- *                       [ecq_codes_words()], bit-identical to what was encoded.  Nothing
+ * ecq_huffman_decode    the inverse: stream_words [stream_len_words] (16-byte aligned),
+ *                       offsets, quarters -> codes [ecq_codes_words()], bit-identical to what was encoded.  Nothing
  *                       beyond stream_len_words is read, whatever the offsets say.  A bit
  *                       pattern that is no word ends its chunk (rest zero) and makes
  *                       ECQ_ERR_SYMBOL pending.
  */
 #define ECQ_HUFFMAN_MAX_LEN 12
 #define ECQ_HUFFMAN_CHUNK 1024
-#define ECQ_HUFFMAN_TABLE_BYTES (4096 * 4 + 4096 * 2)
+#define ECQ_HUFFMAN_TABLE_BYTES (4096 * 4 + 4096 * 4 + 16)
 int ecq_huffman_lengths(const ecq_ctx* ctx, const uint64_t* counts_host, uint8_t* lengths_host);
 uint64_t ecq_huffman_chunks(const ecq_ctx* ctx);
 uint64_t ecq_huffman_stream_bound(const ecq_ctx* ctx, const uint64_t* counts_host,
@@ -238,10 +243,10 @@ int ecq_huffman_tables(ecq_ctx* ctx, const uint8_t* lengths_host, void* tables_d
                        void* cuda_stream);
 int ecq_huffman_encode(ecq_ctx* ctx, const void* tables_dev, const uint32_t* codes,
                        uint32_t* stream_words, uint64_t capacity_words, uint32_t* offsets,
-                       void* cuda_stream);
+                       uint16_t* quarters, void* cuda_stream);
 int ecq_huffman_decode(ecq_ctx* ctx, const void* tables_dev, const uint32_t* stream_words,
-                       uint64_t stream_len_words, const uint32_t* offsets, uint32_t* codes,
-                       void* cuda_stream);
+                       uint64_t stream_len_words, const uint32_t* offsets,
+                       const uint16_t* quarters, uint32_t* codes, void* cuda_stream);
 
 /*
  * One whole iteration from HOST gradients to a HOST result: for every worker

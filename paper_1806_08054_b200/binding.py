@@ -21,7 +21,7 @@ ECQ_ERR_CAPACITY = 7
 ECQ_ERR_SYMBOL = 8
 ECQ_HUFFMAN_MAX_LEN = 12
 ECQ_HUFFMAN_CHUNK = 1024
-ECQ_HUFFMAN_TABLE_BYTES = 4096 * 4 + 4096 * 2
+ECQ_HUFFMAN_TABLE_BYTES = 4096 * 4 + 4096 * 4 + 16
 ECQ_STATIC_SCRATCH_BYTES = 4 << 20
 ECQ_MAX_WORKERS = 64
 ECQ_MAX_WORKERS_TOTAL = 1024
@@ -86,9 +86,9 @@ def lib() -> ctypes.CDLL:
         L.ecq_huffman_stream_bound.restype = u64
         L.ecq_huffman_tables.argtypes = [vp, vp, vp, vp]
         L.ecq_huffman_tables.restype = i32
-        L.ecq_huffman_encode.argtypes = [vp, vp, vp, vp, u64, vp, vp]
+        L.ecq_huffman_encode.argtypes = [vp, vp, vp, vp, u64, vp, vp, vp]
         L.ecq_huffman_encode.restype = i32
-        L.ecq_huffman_decode.argtypes = [vp, vp, vp, u64, vp, vp, vp]
+        L.ecq_huffman_decode.argtypes = [vp, vp, vp, u64, vp, vp, vp, vp]
         L.ecq_huffman_decode.restype = i32
         L.ecq_status.argtypes = [vp, vp]
         L.ecq_status.restype = i32
@@ -311,22 +311,24 @@ def ecq_huffman_tables(ctx: int, lengths, tables: torch.Tensor, stream=None) -> 
 
 
 def ecq_huffman_encode(ctx: int, tables: torch.Tensor, codes: torch.Tensor, stream_words: torch.Tensor,
-                       offsets: torch.Tensor, stream=None) -> None:
-    """Enqueue the entropy coder: ``codes`` -> ``stream_words`` (its size is the capacity)
-    and ``offsets`` (ecq_huffman_chunks() + 1 words)."""
+                       offsets: torch.Tensor, quarters: torch.Tensor, stream=None) -> None:
+    """Enqueue the entropy coder: ``codes`` -> ``stream_words`` (its size is the capacity),
+    ``offsets`` (ecq_huffman_chunks() + 1 words) and ``quarters`` (3 int16 per chunk)."""
     rc = lib().ecq_huffman_encode(ctx, _dev(tables, torch.uint8, "tables"), _dev(codes, torch.int32, "codes"),
                                   _dev(stream_words, torch.int32, "stream_words"), stream_words.numel(),
-                                  _dev(offsets, torch.int32, "offsets"), _stream(stream))
+                                  _dev(offsets, torch.int32, "offsets"),
+                                  _dev(quarters, torch.int16, "quarters"), _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_huffman_encode")
 
 
 def ecq_huffman_decode(ctx: int, tables: torch.Tensor, stream_words: torch.Tensor, offsets: torch.Tensor,
-                       codes: torch.Tensor, stream=None) -> None:
+                       quarters: torch.Tensor, codes: torch.Tensor, stream=None) -> None:
     """Enqueue the inverse of :func:`ecq_huffman_encode`."""
     rc = lib().ecq_huffman_decode(ctx, _dev(tables, torch.uint8, "tables"),
                                   _dev(stream_words, torch.int32, "stream_words"), stream_words.numel(),
-                                  _dev(offsets, torch.int32, "offsets"), _dev(codes, torch.int32, "codes"),
+                                  _dev(offsets, torch.int32, "offsets"),
+                                  _dev(quarters, torch.int16, "quarters"), _dev(codes, torch.int32, "codes"),
                                   _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_huffman_decode")

@@ -538,6 +538,8 @@ int ecq_huffman_tables(ecq_ctx* c, const uint8_t* lengths_host, void* tables_dev
     HuffTables* t = new (std::nothrow) HuffTables;
     if (!t) return ECQ_ERR_ALLOC;
     std::memset(t, 0, sizeof(*t));
+    // one word per 12-bit pattern first: symbol << 4 | length
+    std::vector<uint16_t> single(1u << kHuffMaxLen, 0);
     for (uint32_t k = 0; k < n_sym; ++k) {
         const uint32_t L = lengths_host[k];
         if (!L) continue;
@@ -546,7 +548,27 @@ int ecq_huffman_tables(ecq_ctx* c, const uint8_t* lengths_host, void* tables_dev
         for (uint32_t b = 0; b < L; ++b) rev |= ((word >> (L - 1 - b)) & 1u) << b;
         t->enc[k] = (L << 16) | rev;
         for (uint32_t hi = 0; hi < (1u << (kHuffMaxLen - L)); ++hi)
-            t->dec[(hi << L) | rev] = (uint16_t)((k << 4) | L);
+            single[(hi << L) | rev] = (uint16_t)((k << 4) | L);
+    }
+    // the sender's look-ups take k codes at a time: k*r index bits <= 12, k words <= 24 bits
+    const uint32_t r = c->P.r;
+    uint32_t longest = 1, group = r <= 3 ? 4u : (r <= 6 ? 2u : 1u);
+    for (uint32_t k = 0; k < n_sym; ++k) longest = std::max<uint32_t>(longest, lengths_host[k]);
+    while (group > 1 && group * longest > 24) group /= 2;
+    t->group_syms = group;
+    // then all the words that lie wholly inside the pattern
+    const uint32_t most = std::min<uint32_t>(kHuffDecMaxSyms, 16 / r);
+    for (uint32_t p = 0; p < (1u << kHuffMaxLen); ++p) {
+        uint32_t pos = 0, n = 0, syms = 0, first_len = 0;
+        while (n < most) {
+            const uint16_t e = single[p >> pos];             // the missing high bits read as 0
+            const uint32_t L = e & 15u;
+            if (L == 0 || pos + L > kHuffMaxLen) break;
+            syms |= (uint32_t)(e >> 4) << (n * r);
+            if (n == 0) first_len = L;
+            pos += L; ++n;
+        }
+        t->dec[p] = syms | (n << 16) | (pos << 20) | (first_len << 24);
     }
     // pageable source: the copy is staged before the call returns, so `t` can go
     const cudaError_t e = cudaMemcpyAsync(tables_dev, t, sizeof(*t), cudaMemcpyHostToDevice,
@@ -557,43 +579,51 @@ int ecq_huffman_tables(ecq_ctx* c, const uint8_t* lengths_host, void* tables_dev
 
 int ecq_huffman_encode(ecq_ctx* c, const void* tables_dev, const uint32_t* codes,
                        uint32_t* stream_words, uint64_t capacity_words, uint32_t* offsets,
-                       void* cuda_stream) {
-    if (!c || !tables_dev || !codes || !stream_words || !offsets || !aligned16(tables_dev) ||
-        !aligned16(codes) || !aligned4(stream_words) || !aligned4(offsets))
+                       uint16_t* quarters, void* cuda_stream) {
+    if (!c || !tables_dev || !codes || !stream_words || !offsets || !quarters ||
+        !aligned16(tables_dev) || !aligned16(codes) || !aligned4(stream_words) ||
+        !aligned4(offsets) || (reinterpret_cast<uintptr_t>(quarters) & 1u))
         return ECQ_ERR_ARG;
     const uint32_t n_sym = 2 * c->P.s + 1;
     if (n_sym > kHuffMaxSymbols) return ECQ_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const HuffTables* t = static_cast<const HuffTables*>(tables_dev);
     const uint64_t n_chunks = ecq_huffman_chunks(c);
+    // contiguous segments of chunks, one per CTA, at least one chunk per warp
     uint64_t blocks = (n_chunks + kHuffWarps - 1) / kHuffWarps;
     const uint64_t cap = (uint64_t)c->sm_count * 8;
     if (blocks > cap) blocks = cap;
-    const size_t smem_count = (size_t)n_sym * 4;
-    const size_t smem_write = ((size_t)((n_sym + 31) & ~31u) + kHuffWarps * (kHuffChunkWords + 32)) * 4;
-    huff_count_kernel<<<(uint32_t)blocks, kHuffWarps * 32, smem_count, st>>>(
-        c->P, t, codes, offsets, c->d_status, n_chunks);
-    huff_scan_kernel<<<1, kScanThreads, 0, st>>>(offsets, n_chunks, capacity_words, c->d_status);
-    huff_write_kernel<<<(uint32_t)blocks, kHuffWarps * 32, smem_write, st>>>(
-        c->P, t, codes, offsets, stream_words, n_chunks);
+    const uint64_t seg = (n_chunks + blocks - 1) / blocks;
+    const uint32_t n_seg = (uint32_t)((n_chunks + seg - 1) / seg);
+    // shared memory for the largest group table this code width can have
+    const uint32_t r = c->P.r, k_most = r <= 3 ? 4u : (r <= 6 ? 2u : 1u);
+    const size_t smem_group = (size_t)4 << (k_most * r);
+    const size_t smem_write = smem_group +
+        (size_t)kHuffWarps * (kHuffChunkWords + 32 + 32 * kHuffRowWords) * 4;
+    huff_count_kernel<<<n_seg, kHuffWarps * 32, smem_group, st>>>(
+        c->P, t, codes, offsets, c->d_status, n_chunks, seg);
+    huff_scan_kernel<<<1, kScanThreads, 0, st>>>(offsets, n_chunks, seg, capacity_words, c->d_status);
+    huff_write_kernel<<<n_seg, kHuffWarps * 32, smem_write, st>>>(
+        c->P, t, codes, offsets, quarters, stream_words, n_chunks, seg);
     g_launches.fetch_add(3, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
 }
 
 int ecq_huffman_decode(ecq_ctx* c, const void* tables_dev, const uint32_t* stream_words,
-                       uint64_t stream_len_words, const uint32_t* offsets, uint32_t* codes,
-                       void* cuda_stream) {
-    if (!c || !tables_dev || !stream_words || !offsets || !codes || !aligned16(tables_dev) ||
-        !aligned4(stream_words) || !aligned4(offsets) || !aligned16(codes))
+                       uint64_t stream_len_words, const uint32_t* offsets,
+                       const uint16_t* quarters, uint32_t* codes, void* cuda_stream) {
+    if (!c || !tables_dev || !stream_words || !offsets || !quarters || !codes ||
+        !aligned16(tables_dev) || !aligned16(stream_words) || !aligned4(offsets) ||
+        (reinterpret_cast<uintptr_t>(quarters) & 1u) || !aligned16(codes))
         return ECQ_ERR_ARG;
     const uint32_t n_sym = 2 * c->P.s + 1;
     if (n_sym > kHuffMaxSymbols) return ECQ_ERR_ARG;
     const uint64_t n_chunks = ecq_huffman_chunks(c);
-    uint64_t blocks = (n_chunks + kHuffDecThreads - 1) / kHuffDecThreads;
+    uint64_t blocks = (4 * n_chunks + kHuffDecThreads - 1) / kHuffDecThreads;
     const uint64_t cap = (uint64_t)c->sm_count * 16;
     if (blocks > cap) blocks = cap;
     huff_decode_kernel<<<(uint32_t)blocks, kHuffDecThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        c->P, static_cast<const HuffTables*>(tables_dev), stream_words, offsets, codes, c->d_status,
+        c->P, static_cast<const HuffTables*>(tables_dev), stream_words, offsets, quarters, codes, c->d_status,
         n_chunks, c->n_words, stream_len_words);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;

@@ -53,19 +53,24 @@ class Message:
         pad = 8
         buf = torch.full((cap + 2 * pad,), GUARD, dtype=torch.int32, device="cuda")
         offs = torch.full((self.n_chunks + 1 + 2 * pad,), GUARD, dtype=torch.int32, device="cuda")
-        ecq.ecq_huffman_encode(self.ctx, self.tables, self.codes, buf[pad:pad + cap], offs[pad:pad + self.n_chunks + 1])
+        qts = torch.full((3 * self.n_chunks + 2 * pad,), 0x5A5A, dtype=torch.int16, device="cuda")
+        ecq.ecq_huffman_encode(self.ctx, self.tables, self.codes, buf[pad:pad + cap],
+                               offs[pad:pad + self.n_chunks + 1], qts[pad:pad + 3 * self.n_chunks])
         st = ecq.ecq_status(self.ctx)
-        b, o = u32(buf), u32(offs)
+        b, o, q = u32(buf), u32(offs), qts.cpu().numpy()
         assert np.all(b[:pad] == GUARD) and np.all(b[pad + cap:] == GUARD), "write outside the stream"
         assert np.all(o[:pad] == GUARD) and np.all(o[pad + self.n_chunks + 1:] == GUARD)
+        assert np.all(q[:pad] == 0x5A5A) and np.all(q[pad + 3 * self.n_chunks:] == 0x5A5A)
+        self.quarters = qts[pad:pad + 3 * self.n_chunks]
         return st, buf[pad:pad + cap], offs[pad:pad + self.n_chunks + 1]
 
-    def gpu_decode(self, stream, offsets):
+    def gpu_decode(self, stream, offsets, quarters=None):
         nw = self.codes.numel()
         pad = 8
         out = torch.full((nw + 2 * pad,), GUARD, dtype=torch.int32, device="cuda")
         # 16-byte aligned view: pad is 8 words
-        ecq.ecq_huffman_decode(self.ctx, self.tables, stream, offsets, out[pad:pad + nw])
+        ecq.ecq_huffman_decode(self.ctx, self.tables, stream, offsets,
+                               self.quarters if quarters is None else quarters, out[pad:pad + nw])
         st = ecq.ecq_status(self.ctx)
         o = u32(out)
         assert np.all(o[:pad] == GUARD) and np.all(o[pad + nw:] == GUARD), "write outside the codes"
@@ -83,17 +88,19 @@ def check_against_oracle(m: Message):
     assert kraft(L_lib) <= 1 << 12
     assert cost(m.counts, L_lib) == cost(m.counts, L_or)
     for L in (L_or, L_lib):
-        s_or, o_or = oracle.huffman_encode(m.codes_np, L, n=m.d, s=m.s)
+        s_or, o_or, q_or = oracle.huffman_encode(m.codes_np, L, n=m.d, s=m.s)
         st, stream, offs = m.gpu_encode(L)
         assert st == ecq.ECQ_OK
         assert np.array_equal(u32(offs), o_or), "chunk offsets differ"
+        assert np.array_equal(m.quarters.cpu().numpy().view(np.uint16), q_or), "quarter marks differ"
         assert np.array_equal(u32(stream)[:s_or.size], s_or), "stream differs"
         assert s_or.size <= stream.numel()
         st, back = m.gpu_decode(stream, offs)
         assert st == ecq.ECQ_OK
         assert np.array_equal(back, m.codes_np), "decoded codes differ"
         # and the oracle's decoder reads the GPU's stream
-        assert np.array_equal(oracle.huffman_decode(u32(stream)[:s_or.size], u32(offs), L, n=m.d, s=m.s),
+        assert np.array_equal(oracle.huffman_decode(u32(stream)[:s_or.size], u32(offs),
+                                                    m.quarters.cpu().numpy().view(np.uint16), L, n=m.d, s=m.s),
                               m.codes_np)
 
 
@@ -192,8 +199,8 @@ def test_argument_errors():
         with pytest.raises(ecq.EcqError):             # a word longer than the limit
             ecq.ecq_huffman_tables(m.ctx, [13, 1, 0, 0, 0, 0, 0, 0, 0], m.tables)
         L = ecq.binding.lib()
-        assert L.ecq_huffman_encode(m.ctx, None, None, None, 0, None, None) == ecq.ECQ_ERR_ARG
-        assert L.ecq_huffman_decode(m.ctx, None, None, 0, None, None, None) == ecq.ECQ_ERR_ARG
+        assert L.ecq_huffman_encode(m.ctx, None, None, None, 0, None, None, None) == ecq.ECQ_ERR_ARG
+        assert L.ecq_huffman_decode(m.ctx, None, None, 0, None, None, None, None) == ecq.ECQ_ERR_ARG
     finally:
         m.close()
     big = ecq.ecq_create(1024, 512, 2048, 1.0, 0.9, 1)      # 4097 levels: beyond the coder
