@@ -225,3 +225,59 @@ def test_resnet50_sized_message_bits_per_entry():
         assert payload < 0.8 * w.d * ecq.ecq_code_bits(m.ctx)
     finally:
         m.close()
+
+
+def test_lm_350m_sized_message_on_sampled_chunks():
+    # full benchmark size: the oracle codes sampled runs of chunks (a chunk's stream depends
+    # only on its own entries); offsets and quarter marks are checked there, the round trip
+    # over the whole message on the device
+    w = wl.WORKLOADS["lm_350m"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * w.d:
+        pytest.skip("needs %.0f GB of free device memory" % (12 * w.d / 1e9))
+    ctx = ecq.ecq_create(w.d, w.bucket, w.s, 1.0, 0.9, SEED)
+    try:
+        r = ecq.ecq_code_bits(ctx)
+        grad = wl.gradient(w, 0, 0, "cuda")
+        err = torch.zeros(w.d, device="cuda")
+        codes = torch.zeros(ecq.ecq_codes_words(ctx), dtype=torch.int32, device="cuda")
+        scales = torch.zeros(ecq.ecq_num_buckets(ctx), device="cuda")
+        ecq.ecq_encode(ctx, 0, 0, grad, err, codes, scales)
+        del grad, err
+        counts_dev = torch.zeros(2 * w.s + 1, dtype=torch.int64, device="cuda")
+        ecq.ecq_code_histogram(ctx, codes, counts_dev)
+        counts = counts_dev.cpu().numpy().astype(np.uint64)
+        assert int(counts.sum()) == w.d
+        L = oracle.huffman_lengths(counts, max_len=12)
+        n_chunks = ecq.ecq_huffman_chunks(ctx)
+        cap = ecq.ecq_huffman_stream_bound(ctx, counts, L)
+        tables = torch.zeros(ecq.ECQ_HUFFMAN_TABLE_BYTES, dtype=torch.uint8, device="cuda")
+        stream = torch.zeros(cap, dtype=torch.int32, device="cuda")
+        offsets = torch.zeros(n_chunks + 1, dtype=torch.int32, device="cuda")
+        quarters = torch.zeros(3 * n_chunks, dtype=torch.int16, device="cuda")
+        ecq.ecq_huffman_tables(ctx, L, tables)
+        ecq.ecq_huffman_encode(ctx, tables, codes, stream, offsets, quarters)
+        assert ecq.ecq_status(ctx) == ecq.ECQ_OK
+        off = u32(offsets).astype(np.int64)
+        assert off[0] == 0 and np.all(np.diff(off) >= 0) and off[-1] <= cap
+        # the whole stream is as long as the counts say, up to the padding of each chunk
+        payload = cost(counts, L)
+        assert payload <= 32 * off[-1] < payload + 32 * n_chunks
+        rng = np.random.default_rng(7)
+        starts = [0, n_chunks - 40] + [int(x) for x in rng.integers(0, n_chunks - 40, size=4)]
+        for c0 in starts:
+            c1 = min(c0 + 40, n_chunks)
+            lo, hi = c0 * 1024, min(c1 * 1024, w.d)
+            piece = u32(codes[c0 * 32 * r: -(-hi * r // 32)])
+            s_or, o_or, q_or = oracle.huffman_encode(piece, L, n=hi - lo, s=w.s)
+            assert np.array_equal(off[c0:c1 + 1] - off[c0], o_or.astype(np.int64))
+            assert np.array_equal(u32(stream[off[c0]:off[c1]]), s_or)
+            assert np.array_equal(quarters[3 * c0:3 * c1].cpu().numpy().view(np.uint16), q_or)
+        back = torch.zeros_like(codes)
+        ecq.ecq_huffman_decode(ctx, tables, stream, offsets, quarters, back)
+        assert ecq.ecq_status(ctx) == ecq.ECQ_OK
+        assert torch.equal(back, codes)
+    finally:
+        ecq.ecq_destroy(ctx)
+        wl.clear_cache()
+        torch.cuda.empty_cache()

@@ -448,6 +448,24 @@ def test_config5_lm_350m_sweep(bucket, s):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("s", [3, 7, 127])
+def test_code_width_matched_levels_on_lm_350m(s):
+    # the same width-matched quantisers at the benchmark's full size (B = 512, 4 workers)
+    w = wl.with_codec(wl.WORKLOADS["lm_350m"], 512, s)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 4 * w.d * 4 * 3.5:
+        pytest.skip("needs %.0f GB of free device memory" % (4 * w.d * 4 * 3.5 / 1e9))
+    cache = {}
+
+    def grads(p, t):
+        if (p, t) not in cache:
+            cache[(p, t)] = wl.gradient(w, p, t, "cuda")
+        return cache[(p, t)]
+    _sampled_config(w, steps=1, W=4, grads=grads)
+    cache.clear()
+    torch.cuda.empty_cache()
+
+
 def test_code_width_matched_levels_on_resnet50():
     # the quantiser whose 2s+1 levels exactly fill b bits: s = 2^(b-1) - 1
     base = wl.WORKLOADS["resnet50"]
