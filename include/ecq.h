@@ -14,7 +14,7 @@
  *     is the default stream) and the call returns without synchronising,
  *     unless stated otherwise.
  *   - `grad`, `err`, `out`, `codes` must be 16-byte aligned; `scales` 4-byte.
- *   - A context is immutable after creation (except ecq_set_error_mode) and may
+ *   - A context is immutable after creation (except ecq_set_error_mode, ecq_set_norm and ecq_set_decode_plan) and may
  *     be used from several host threads on different streams.
  *   - Inputs must be finite.  A bucket whose compensated values contain NaN or
  *     Inf is sent as all-zero levels with scale 0, its accumulator entries are
@@ -97,6 +97,24 @@ int ecq_set_error_mode(ecq_ctx* ctx, int mode);
  * The receiver side is the same for both.
  */
 int ecq_set_norm(ecq_ctx* ctx, int norm);
+
+/*
+ * Choose how the receiver side (Eq. 4; ecq_decode_mean and ecq_decode_mean_update) is
+ * launched.  The result does not depend on the choice: every kernel sums the W terms of an
+ * output in ascending worker order with one fused multiply-add per term.
+ *   kernel    ECQ_DECODE_AUTO (default): by shape and length;
+ *             ECQ_DECODE_WARP: tiles of 1024 outputs, every warp copies its own code words;
+ *             ECQ_DECODE_RING: tiles of 16384 outputs, one bulk copy per (tile, worker)
+ *             shared by the CTA (what AUTO takes for long vectors).
+ *             A shape that a kernel does not cover (bucket not a power of two, r > 9, more
+ *             than bucket/4 workers for buckets under 1024) falls through to the next one.
+ *   max_ctas  upper limit on the CTAs of a launch; 0 = fill the device.
+ * ECQ_ERR_ARG on an unknown kernel.
+ */
+#define ECQ_DECODE_AUTO 0
+#define ECQ_DECODE_WARP 1
+#define ECQ_DECODE_RING 2
+int ecq_set_decode_plan(ecq_ctx* ctx, int kernel, uint32_t max_ctas);
 
 /* r = ceil(log2(2s+1)): bits per entry (paragraph after Eq. 9). */
 uint32_t ecq_code_bits(const ecq_ctx* ctx);

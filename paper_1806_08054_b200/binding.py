@@ -54,6 +54,8 @@ def lib() -> ctypes.CDLL:
         L.ecq_set_error_mode.restype = i32
         L.ecq_set_norm.argtypes = [vp, i32]
         L.ecq_set_norm.restype = i32
+        L.ecq_set_decode_plan.argtypes = [vp, i32, ctypes.c_uint32]
+        L.ecq_set_decode_plan.restype = i32
         L.ecq_code_bits.argtypes = [vp]
         L.ecq_code_bits.restype = u32
         L.ecq_num_buckets.argtypes = [vp]
@@ -142,6 +144,16 @@ def ecq_set_norm(ctx: int, norm: int) -> None:
     rc = lib().ecq_set_norm(ctx, norm)
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_set_norm")
+
+
+ECQ_DECODE_AUTO, ECQ_DECODE_WARP, ECQ_DECODE_RING = 0, 1, 2
+
+
+def ecq_set_decode_plan(ctx: int, kernel: int = ECQ_DECODE_AUTO, max_ctas: int = 0) -> None:
+    """Which receiver kernel a launch takes and how many CTAs at most (0: fill the device)."""
+    rc = lib().ecq_set_decode_plan(ctx, kernel, max_ctas)
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_set_decode_plan")
 
 
 def ecq_code_bits(ctx: int) -> int:

@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libecq.so")
 SOURCES = ["ecq_api.cu"]
-HEADERS = ["ecq_common.cuh", "ecq_encode.cuh", "ecq_decode.cuh", "ecq_stats.cuh", "ecq_entropy.cuh"]
+HEADERS = ["ecq_common.cuh", "ecq_encode.cuh", "ecq_decode.cuh", "ecq_decode_ring.cuh", "ecq_stats.cuh", "ecq_entropy.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -16,6 +16,7 @@
 #include "../../include/ecq.h"
 #include "ecq_common.cuh"
 #include "ecq_decode.cuh"
+#include "ecq_decode_ring.cuh"
 #include "ecq_encode.cuh"
 #include "ecq_stats.cuh"
 #include "ecq_entropy.cuh"
@@ -57,6 +58,8 @@ struct ecq_ctx {
     uint32_t* d_status;
     uint32_t* h_status;          // pinned
     bool tiled_ok;               // bucket is a power of two <= 4096
+    int decode_kernel;           // ECQ_DECODE_AUTO / _WARP / _RING (ecq_set_decode_plan)
+    uint32_t decode_max_ctas;    // 0: fill the device
     // lazily created by ecq_step_host
     std::mutex host_mu;
     cudaStream_t copy_stream;
@@ -246,8 +249,45 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, Decode
     uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
     const uint32_t want = (n_tiles + kDecWarps - 1) / kDecWarps;
     if (grid > want) grid = want;
+    if (c->decode_max_ctas && grid > c->decode_max_ctas) grid = c->decode_max_ctas;
     kern<<<grid, kDecWarps * 32, L::kSmem, st>>>(c->P, W, tab, out, n_tiles, c->n_words, w_recip,
                                                  w_pow2, 0x4B000000u, sl);
+    return true;
+}
+
+// Ring decode (long vectors): returns false when the shape is not covered or the vector is
+// too short to give every CTA a few tiles (caller goes on to the warp-tiled kernel).
+template <int R, bool CARRY>
+bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeOut out,
+                        cudaStream_t st, float w_recip, int w_pow2, DecodeSlice sl) {
+    using L = DecodeRing<R>;
+    const uint32_t B = c->P.bucket;
+    const uint64_t n_subs64 = c->P.d / kDecTileElems;
+    if ((B & (B - 1)) != 0 || n_subs64 == 0 || n_subs64 > 0xFFFFFFFFull) return false;
+    const uint32_t gsz = B >= 1024 ? 32 : B / 32;
+    if (W > (uint32_t)kDecAreg * gsz) return false;
+    const uint64_t n_tiles = (n_subs64 + kRingSubs - 1) / kRingSubs;
+    if (n_tiles * W > 0xFFFFFFFFull) return false;
+    static std::once_flag once[16];
+    static int occ[16];
+    const int dev = c->device & 15;
+    auto kern = decode_ring_kernel<R, CARRY>;
+    std::call_once(once[dev], [&] {
+        int o = 0;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmem) ==
+                cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kRingWarps * 32, L::kSmem) ==
+                cudaSuccess)
+            occ[dev] = o;
+    });
+    if (occ[dev] <= 0) return false;
+    uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
+    if (c->decode_kernel == ECQ_DECODE_AUTO && n_tiles < (uint64_t)kRingMinTilesPerCta * grid)
+        return false;
+    if (c->decode_max_ctas && grid > c->decode_max_ctas) grid = c->decode_max_ctas;
+    if (grid > n_tiles) grid = (uint32_t)n_tiles;
+    kern<<<grid, kRingWarps * 32, L::kSmem, st>>>(c->P, W, tab, out, (uint32_t)n_subs64, c->n_words,
+                                                  w_recip, w_pow2, 0x4B000000u, sl, c->d_status);
     return true;
 }
 
@@ -259,7 +299,15 @@ int decode_launch(ecq_ctx* c, uint32_t W, uint32_t w_all, const MessageTable& ta
     const float w_recip = 1.0f / (float)w_all;
     const DecodeSlice sl{(float)w_all, first, last};
     bool done = false;
-    switch (c->P.r) {
+    if (c->decode_kernel != ECQ_DECODE_WARP) switch (c->P.r) {
+#define ECQ_CASE(R) case R: done = (first && last)                                                      \
+            ? launch_decode_ring<R, false>(c, W, tab, out, st, w_recip, w_pow2, sl)                      \
+            : launch_decode_ring<R, true>(c, W, tab, out, st, w_recip, w_pow2, sl); break;
+        ECQ_CASE(2) ECQ_CASE(3) ECQ_CASE(4) ECQ_CASE(5) ECQ_CASE(6) ECQ_CASE(7) ECQ_CASE(8) ECQ_CASE(9)
+#undef ECQ_CASE
+        default: break;
+    }
+    if (!done) switch (c->P.r) {
 #define ECQ_CASE(R) case R: done = (first && last)                                                      \
             ? launch_decode_tiled<R, false>(c, W, tab, out, st, w_recip, w_pow2, sl)                     \
             : launch_decode_tiled<R, true>(c, W, tab, out, st, w_recip, w_pow2, sl); break;
@@ -335,6 +383,8 @@ int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels, floa
     c->nb = (d + bucket - 1) / bucket;
     c->n_words = (d * P.r + 31) / 32;
     c->tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= kMaxTiledBucket;
+    c->decode_kernel = ECQ_DECODE_AUTO;
+    c->decode_max_ctas = 0;
     c->host_ready = false;
     c->d_status = nullptr; c->h_status = nullptr;
     if (cudaGetDevice(&c->device) != cudaSuccess ||
@@ -368,6 +418,13 @@ void ecq_destroy(ecq_ctx* c) {
 int ecq_set_error_mode(ecq_ctx* c, int mode) {
     if (!c || (mode != 0 && mode != 1)) return ECQ_ERR_ARG;
     c->P.mode = mode;
+    return ECQ_OK;
+}
+
+int ecq_set_decode_plan(ecq_ctx* c, int kernel, uint32_t max_ctas) {
+    if (!c || kernel < ECQ_DECODE_AUTO || kernel > ECQ_DECODE_RING) return ECQ_ERR_ARG;
+    c->decode_kernel = kernel;
+    c->decode_max_ctas = max_ctas;
     return ECQ_OK;
 }
 
@@ -790,6 +847,8 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
     c.nb = (d + bucket - 1) / bucket;
     c.n_words = (d * P.r + 31) / 32;
     c.tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= kMaxTiledBucket;
+    c.decode_kernel = ECQ_DECODE_AUTO;
+    c.decode_max_ctas = 0;
     c.host_ready = false;
     c.h_status = nullptr;
 

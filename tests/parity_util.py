@@ -27,13 +27,15 @@ def close(x: np.ndarray, y: np.ndarray) -> bool:
 class GpuCodec:
     """Owns a context and the per-worker device buffers of one configuration."""
 
-    def __init__(self, d, bucket, s, alpha, beta, seed, W, mode=0, norm=0):
+    def __init__(self, d, bucket, s, alpha, beta, seed, W, mode=0, norm=0, decode_plan=None):
         self.d, self.bucket, self.s, self.W = d, bucket, s, W
         self.ctx = ecq.ecq_create(d, bucket, s, alpha, beta, seed)
         if mode:
             ecq.ecq_set_error_mode(self.ctx, mode)
         if norm:
             ecq.ecq_set_norm(self.ctx, norm)
+        if decode_plan is not None:
+            ecq.ecq_set_decode_plan(self.ctx, *decode_plan)
         self.r = ecq.ecq_code_bits(self.ctx)
         self.nb = ecq.ecq_num_buckets(self.ctx)
         self.nw = ecq.ecq_codes_words(self.ctx)
@@ -86,12 +88,12 @@ def codes_np(t: torch.Tensor) -> np.ndarray:
 
 
 def full_parity(d, bucket, s, alpha, beta, seed, W, steps, grad_fn, mode=0, err0=None,
-                expect_status=ecq.ECQ_OK, check_decode=True, batch=False, norm=0):
+                expect_status=ecq.ECQ_OK, check_decode=True, batch=False, norm=0, decode_plan=None):
     """Element-by-element comparison over whole vectors.
 
     ``grad_fn(worker, step)`` returns a float32 CUDA tensor of d entries.
     """
-    gpu = GpuCodec(d, bucket, s, alpha, beta, seed, W, mode, norm)
+    gpu = GpuCodec(d, bucket, s, alpha, beta, seed, W, mode, norm, decode_plan)
     try:
         h_or = [np.zeros(d, np.float32) for _ in range(W)]
         if err0 is not None:
