@@ -241,6 +241,8 @@ def main():
     ap.add_argument("--bucket", type=int, default=0)
     ap.add_argument("--levels", type=int, default=0)
     ap.add_argument("--workers", type=int, default=0, help="override W (smaller runs)")
+    ap.add_argument("--decode-kernel", default="auto", choices=["auto", "warp", "ring"],
+                    help="receiver kernel (ecq_set_decode_plan); auto = the library's choice")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -272,6 +274,8 @@ def main():
 
     d, W = w.d, w.W
     ctx = ecq.ecq_create(d, w.bucket, w.s, w.alpha, w.beta, wl.CODEC_SEED)
+    ecq.ecq_set_decode_plan(ctx, {"auto": ecq.ECQ_DECODE_AUTO, "warp": ecq.ECQ_DECODE_WARP,
+                                  "ring": ecq.ECQ_DECODE_RING}[args.decode_kernel], 0)
     r = ecq.ecq_code_bits(ctx)
     nw, nb = ecq.ecq_codes_words(ctx), ecq.ecq_num_buckets(ctx)
     enc_bytes, dec_bytes = step_bytes(w)
@@ -403,7 +407,7 @@ def main():
                                 "entropy-coded on other workloads (context only)"},
             # the decode kernel's own bound: one logic instruction per code on the ALU pipe
             # (16 lanes per clock per SM sub-partition)
-            "decode_roofline": {"kernel": "decode_tiled_kernel", "bound": "alu",
+            "decode_roofline": {"kernel": "decode kernel (%s)" % args.decode_kernel, "bound": "alu",
                                 "achieved": W * d * args.steps / (dec_ms * 1e-3) / 1e12,
                                 "peak": 148 * 4 * 16 * 1.965e9 / 1e12, "unit": "Tcodes/s",
                                 "frac": (W * d * args.steps / (dec_ms * 1e-3)) / (148 * 4 * 16 * 1.965e9),

@@ -104,10 +104,11 @@ int ecq_set_norm(ecq_ctx* ctx, int norm);
  * output in ascending worker order with one fused multiply-add per term.
  *   kernel    ECQ_DECODE_AUTO (default): by shape and length;
  *             ECQ_DECODE_WARP: tiles of 1024 outputs, every warp copies its own code words;
- *             ECQ_DECODE_RING: tiles of 16384 outputs, one bulk copy per (tile, worker)
- *             shared by the CTA (what AUTO takes for long vectors).
+ *             ECQ_DECODE_RING: tiles of 30720 outputs, one bulk copy per (tile, worker)
+ *             shared by the CTA (what AUTO takes for long vectors with r <= 8).
  *             A shape that a kernel does not cover (bucket not a power of two, r > 9, more
- *             than bucket/4 workers for buckets under 1024) falls through to the next one.
+ *             than bucket/4 workers for buckets under 1024; for RING also `out` or
+ *             `params` not 32-byte aligned) falls through to the next one.
  *   max_ctas  upper limit on the CTAs of a launch; 0 = fill the device.
  * ECQ_ERR_ARG on an unknown kernel.
  */

@@ -14,6 +14,7 @@ from __future__ import annotations
 import ctypes
 import os
 import subprocess
+import threading
 from typing import Optional, Sequence
 
 import numpy as np
@@ -27,20 +28,29 @@ STATUS_NONFINITE = 1
 
 def build(force: bool = False) -> str:
     """Compile the oracle (no optimisation that changes fp32 results)."""
-    if force or not os.path.exists(_LIB) or \
-            os.path.getmtime(_LIB) < max(os.path.getmtime(p) for p in _SRCS):
-        tmp = _LIB + ".tmp.%d" % os.getpid()
-        subprocess.check_call([
-            "g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math",
-            "-shared", "-fPIC", "-o", tmp] + _SRCS)
-        os.replace(tmp, _LIB)
+    with _build_lock:          # callers may be pool threads that all find the library missing
+        if force or not os.path.exists(_LIB) or \
+                os.path.getmtime(_LIB) < max(os.path.getmtime(p) for p in _SRCS):
+            tmp = _LIB + ".tmp.%d.%d" % (os.getpid(), threading.get_ident())
+            subprocess.check_call([
+                "g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math",
+                "-shared", "-fPIC", "-o", tmp] + _SRCS)
+            os.replace(tmp, _LIB)
     return _LIB
 
 
+_build_lock = threading.Lock()
+_load_lock = threading.Lock()
 _lib = None
 
 
 def _load():
+    global _lib
+    with _load_lock:
+        return _load_locked()
+
+
+def _load_locked():
     global _lib
     if _lib is None:
         lib = ctypes.CDLL(build())

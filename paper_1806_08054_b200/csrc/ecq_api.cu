@@ -266,6 +266,9 @@ bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeO
     if ((B & (B - 1)) != 0 || n_subs64 == 0 || n_subs64 > 0xFFFFFFFFull) return false;
     const uint32_t gsz = B >= 1024 ? 32 : B / 32;
     if (W > (uint32_t)kDecAreg * gsz) return false;
+    // the kernel stores 32 bytes at a time
+    if ((reinterpret_cast<uintptr_t>(out.out) & 31u) || (reinterpret_cast<uintptr_t>(out.params) & 31u))
+        return false;
     const uint64_t n_tiles = (n_subs64 + kRingSubs - 1) / kRingSubs;
     if (n_tiles * W > 0xFFFFFFFFull) return false;
     static std::once_flag once[16];
@@ -276,17 +279,18 @@ bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeO
         int o = 0;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmem) ==
                 cudaSuccess &&
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kRingWarps * 32, L::kSmem) ==
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kRingThreads, L::kSmem) ==
                 cudaSuccess)
             occ[dev] = o;
     });
     if (occ[dev] <= 0) return false;
     uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
-    if (c->decode_kernel == ECQ_DECODE_AUTO && n_tiles < (uint64_t)kRingMinTilesPerCta * grid)
+    if (c->decode_kernel == ECQ_DECODE_AUTO &&
+        (n_tiles < (uint64_t)kRingMinTilesPerCta * grid || R > kRingMaxAutoBits))
         return false;
     if (c->decode_max_ctas && grid > c->decode_max_ctas) grid = c->decode_max_ctas;
     if (grid > n_tiles) grid = (uint32_t)n_tiles;
-    kern<<<grid, kRingWarps * 32, L::kSmem, st>>>(c->P, W, tab, out, (uint32_t)n_subs64, c->n_words,
+    kern<<<grid, kRingThreads, L::kSmem, st>>>(c->P, W, tab, out, (uint32_t)n_subs64, c->n_words,
                                                   w_recip, w_pow2, 0x4B000000u, sl, c->d_status);
     return true;
 }

@@ -2,15 +2,14 @@
 // Algorithm 1, "compute global gradients"), with the code words brought in by bulk copies
 // that a whole CTA shares.
 //
-// A CTA tile is 16 sub-tiles of 1024 outputs.  Warp k owns sub-tiles k and k + 8; a lane
-// owns one run of 32 consecutive outputs ("row") in each, whose codes are R whole words.
-//   * unit (tile, worker) = the worker's code words of the tile, R * 2048 contiguous
-//     bytes: ONE bulk copy into a ring of stages, signalled on the stage's mbarrier.  A warp
-//     that has copied its rows to registers counts itself off the stage; the warp that
-//     counts last refills the stage at once with the unit `stages` further on, so no warp
-//     is the producer and the ring stays full whichever warp runs ahead.  Per unit a warp
-//     spends a wait, two shared loads and one atomic on data movement instead of issuing
-//     and tracking its own copies;
+// One CTA per SM: 15 consumer warps and one producer warp.  A CTA tile is 30 sub-tiles of
+// 1024 outputs.  Consumer warp k owns sub-tiles k and k + 15; a lane owns one run of 32
+// consecutive outputs ("row") in each, whose codes are R whole words.
+//   * unit (tile, worker) = the worker's code words of the tile, R * 3840 contiguous
+//     bytes: ONE bulk copy into a ring of stages, signalled on the stage's "full"
+//     mbarrier.  Lane 0 of the producer warp issues the copies in order, each as soon as
+//     the 15 consumer warps have handed its stage back on the "empty" mbarrier.  Per unit a
+//     consumer warp spends a wait, two shared loads and an arrive on data movement;
 //   * the two rows of a lane travel as the two halves of packed fp32x2 registers:
 //     (word_A & field, word_B & field) | 2^23 exponent bits is (2^23 + c 2^p) for both rows,
 //     one packed subtract leaves ((c - s) 2^p), one packed multiply-add with the pair of
@@ -18,37 +17,42 @@
 //     acc <- fma(q_w, a_w, acc) is the one Eq. 4 writes out, in ascending w;
 //   * level steps a_w = scale_w / s of the next tile are fetched with 4-byte asynchronous
 //     copies while this tile is summed;
-//   * means leave through a swizzled staging buffer so that stores to `out` are coalesced.
+//   * a lane stores its rows with 32-byte stores (whole sectors), so the means need no
+//     transposition; `out` and `params` must be 32-byte aligned for this kernel.
 #pragma once
 
 #include "ecq_decode.cuh"
 
 namespace ecq {
 
-#ifndef ECQ_RING_WARPS
-#define ECQ_RING_WARPS 8
-#endif
-constexpr int kRingWarps = ECQ_RING_WARPS;
+// 15 consumer warps and the producer warp make 512 threads, which leaves a thread 128 registers
+constexpr int kRingWarps = 15;
+constexpr int kRingThreads = (kRingWarps + 1) * 32;
 constexpr int kRingSubs = 2 * kRingWarps;                       // sub-tiles per CTA tile
-constexpr int kRingTileElems = kRingSubs * kDecTileElems;       // 16384 outputs
-// shorter vectors leave the CTAs with too uneven a share of these large tiles
-constexpr int kRingMinTilesPerCta = 1;
+constexpr int kRingTileElems = kRingSubs * kDecTileElems;       // 30720 outputs
+// What the automatic choice asks for: shorter vectors leave the CTAs with too uneven a share
+// of these large tiles (measured: 7 % slower than the warp-tiled kernel at 5.6 tiles per CTA,
+// 7 % faster at 13, 10 % faster at 78), and at r = 9 the receiver is bound by HBM, not by
+// instruction issue, where the warp-tiled kernel's deeper private rings do better.
+constexpr int kRingMinTilesPerCta = 12;
+constexpr int kRingMaxAutoBits = 8;
 
 template <int R> struct DecodeRing {
     static constexpr int kUnitBytes = R * 128 * kRingSubs;
-    // about 36 KB of copies in flight per CTA, sized so that two CTAs share an SM up to r = 8
-    static constexpr int kStagesRaw = 36864 / kUnitBytes + 1;
-    static constexpr int kStages = kStagesRaw < 3 ? 3 : (kStagesRaw > 8 ? 8 : kStagesRaw);
     // whole fields below bit 23 of a word; chosen so that the fewest groups need a shift
     static constexpr int kFit = R == 2 ? 8 : R == 3 ? 7 : R == 4 ? 4 : 23 / R;
-    static constexpr int kBarBytes = 256;                        // 2 * kStages mbarriers, then the abort flag
-    static constexpr int kStageBytes = 4096;                     // per warp: 32 x 32 floats
+    // full mbarriers at 0, empty ones at 128, abort flag at 256, units issued at 260
+    static constexpr int kBarBytes = 512;
     static constexpr int kATabBytes = kDecAreg * 32 * 8;         // per warp: (a_A, a_B) pairs
     static constexpr int kRawBytes = kDecAreg * 32 * 8;          // per warp: raw scales, rows A and B
-    static constexpr int kWarpBytes = kStageBytes + kATabBytes + kRawBytes;
+    static constexpr int kWarpBytes = kATabBytes + kRawBytes;
+    // the ring takes what one CTA per SM can have
+    static constexpr int kStagesRaw = (232448 - 1024 - kBarBytes - kRingWarps * kWarpBytes) / kUnitBytes;
+    static constexpr int kStages = kStagesRaw > 12 ? 12 : kStagesRaw;
     static constexpr int kRingOff = kBarBytes;
     static constexpr int kWarpOff = kRingOff + kStages * kUnitBytes;
     static constexpr int kSmem = kWarpOff + kRingWarps * kWarpBytes;
+    static_assert(kStages >= 3 && 8 * kStages <= 128, "ring depth fits the barrier area");
 };
 
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
@@ -65,66 +69,54 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* gsrc, uin
         : "memory");
 }
 
-__device__ __forceinline__ uint32_t atom_add_acq_rel_shared(uint32_t a, uint32_t v) {
-    uint32_t old;
-    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(a), "r"(v) : "memory");
-    return old;
+__device__ __forceinline__ void stg256(float* p, const float (&v)[8]) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                 : "memory");
 }
-__device__ __forceinline__ void st_shared_u32(uint32_t a, uint32_t v) {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+__device__ __forceinline__ void ldg256(const float* p, float (&v)[8]) {
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p)
+                 : "memory");
+}
+// eight consecutive means: to `out` (may be null) and, for the fused model update, into `params`
+__device__ __forceinline__ void emit8(const DecodeOut& o, uint64_t i, const float (&v)[8]) {
+    if (o.params) {
+        float p[8];
+        ldg256(o.params + i, p);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) p[k] = __fmaf_rn(o.neg_eta, v[k], p[k]);
+        stg256(o.params + i, p);
+    }
+    if (o.out) stg256(o.out + i, v);
 }
 __device__ __forceinline__ void lds32(uint32_t a, uint32_t& x) {
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x) : "r"(a));
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x) : "r"(a) : "memory");
 }
 __device__ __forceinline__ void lds64(uint32_t a, uint32_t& x, uint32_t& y) {
-    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(a));
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(x), "=r"(y) : "r"(a) : "memory");
 }
 __device__ __forceinline__ void lds128(uint32_t a, uint32_t& x, uint32_t& y, uint32_t& z, uint32_t& w) {
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(a));
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(a) : "memory");
 }
 
+// What one consumer warp does: its two rows of every tile of the CTA.
 template <int R, bool CARRY>
-__global__ void __launch_bounds__(kRingWarps * 32, 2)
-decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
-                   const DecodeOut dst, const uint32_t n_subs, const uint64_t n_words,
-                   const float w_recip, const int w_pow2, const uint32_t exp23_bits,
-                   const DecodeSlice sl, uint32_t* status) {
+__device__ __forceinline__ void decode_ring_consumer(
+        const CodecParams& P, const uint32_t W, const MessageTable& tab, const DecodeOut& dst,
+        const uint32_t n_subs, const float w_recip, const int w_pow2, const uint32_t exp23_bits,
+        const bool first, const bool last, const float w_total, const uint32_t my_tiles,
+        const int warp, const int lane, uint8_t* dsm, uint32_t* status) {
     using L = DecodeRing<R>;
-    const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
-    const float w_total = CARRY ? sl.w_total : (float)W;
     constexpr int S = L::kStages;
     constexpr int FIT = L::kFit;
     constexpr uint32_t mask = (1u << R) - 1u;
-    extern __shared__ __align__(128) uint8_t dsm[];
     const uint32_t sm0 = smem_u32(dsm);
-    // [0, 64) full mbarriers; [64, 96) warps still to read a stage; [96, 128) copies issued
-    // into a stage so far; [128] abort flag
-    const uint32_t bar_full = sm0, cnt_u32 = sm0 + 64;
-    uint32_t* const s_issued = reinterpret_cast<uint32_t*>(dsm + 96);
-    volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 128);
-    static_assert(S <= 8 && L::kBarBytes >= 132, "barriers, counters and flag fit their area");
-    const int lane = threadIdx.x & 31;
-    // broadcast from lane 0 so that the compiler knows the value is warp-uniform
-    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
-    uint8_t* const stage = dsm + L::kWarpOff + warp * L::kWarpBytes;
-    float2* const a_tab = reinterpret_cast<float2*>(stage + L::kStageBytes);
-    float* const raw = reinterpret_cast<float*>(stage + L::kStageBytes + L::kATabBytes);
-
-    const uint32_t n_tiles = (n_subs + kRingSubs - 1) / kRingSubs;
-    const uint32_t my_tiles =
-        blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    const uint32_t n_units = my_tiles * W;                          // < 2^32: checked by the host
-
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < S; ++i) {
-            mbar_init(bar_full + 8 * i, 1);
-            reinterpret_cast<uint32_t*>(dsm + 64)[i] = 0;
-            s_issued[i] = 0;
-        }
-        *s_abort = 0;
-        fence_mbar_init();
-    }
-    __syncthreads();
+    const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
+    volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 256);
+    float2* const a_tab = reinterpret_cast<float2*>(dsm + L::kWarpOff + warp * L::kWarpBytes);
+    float* const raw = reinterpret_cast<float*>(dsm + L::kWarpOff + warp * L::kWarpBytes + L::kATabBytes);
 
     // lanes that share a bucket: gsz consecutive lanes (all 32 from 1024 entries up); a_tab
     // holds, per group of lanes, (a_w of row A, a_w of row B) for w < W (W <= kDecAreg * gsz)
@@ -147,17 +139,6 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
     // logic instruction takes one immediate, and the field mask is it
     const uint64_t magic2 = ((uint64_t)exp23_bits << 32) | exp23_bits;
 
-    // ---- one bulk copy: the code words of (tile, worker w) into stage `slot` ----
-    auto issue_unit = [&](uint32_t tile, uint32_t w, uint32_t slot) {
-        const uint32_t subs = min((uint32_t)kRingSubs, n_subs - tile * kRingSubs);
-        const uint32_t bytes = subs * (R * 128);
-        const uint32_t bar = bar_full + 8 * slot;
-        s_issued[slot] += 1;
-        mbar_arrive_expect_tx(bar, bytes);
-        bulk_load_1d(sm0 + L::kRingOff + slot * L::kUnitBytes,
-                     tab.codes[w] + (uint64_t)tile * (R * 32 * kRingSubs), bytes, bar);
-    };
-
     // ---- raw scales of a tile's buckets: worker k*gsz + gl of my group, rows A and B ----
     auto fetch_scales = [&](uint32_t tile) {
 #pragma unroll
@@ -175,79 +156,57 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         }
         cp_async_commit();
     };
-
-    bool ok = true;
-    // (r_tile, r_w): the unit `S` units after the one a warp takes next, i.e. the refill of its stage
-    uint32_t r_tile = blockIdx.x, r_w = 0;
-    for (uint32_t u = 0; u < (uint32_t)S; ++u) {
-        if (threadIdx.x == 0 && u < n_units) issue_unit(r_tile, r_w, u);
-        if (++r_w == W) { r_w = 0; r_tile += gridDim.x; }
-    }
     if (my_tiles) fetch_scales(blockIdx.x);
 
-    // consumer state: ring offset and phase of the next unit to read, units still to take
-    uint32_t c_off = 0, c_par = 0, c_left = n_units;
+    // ring position of the next unit: stage offset, its barriers' offset, phase
+    uint32_t c_off = 0, c_bar = 0, c_par = 0, held_bar = 0;
     const uint32_t my_off = sm0 + L::kRingOff + warp * (R * 128) + lane * (R * 4);
-    uint32_t cwa[2][R];
-    // waits for the next unit, copies my two rows' words to registers, frees the stage
-    auto take_unit = [&](uint32_t (&dstw)[2][R]) -> bool {
-        const uint32_t slot = c_off / L::kUnitBytes;
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_full + slot * 8, c_par))) return false;
+    uint32_t cw[2][R];
+    // Waits for the next unit and copies my two rows' words to registers.  The stage is handed
+    // back only after the words have been used (release_unit): the loads have then certainly
+    // completed, which an arrive issued right behind them does not wait for.  Loading at the
+    // top of every turn keeps the words out of the loop-carried state (carrying them from the
+    // end of the previous turn cost 20 register moves a unit).
+    auto take_unit = [&]() -> bool {
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_full + c_bar, c_par))) return false;
 #pragma unroll
         for (int row = 0; row < 2; ++row) {
             const uint32_t src = my_off + c_off + row * (kRingWarps * R * 128);
             if constexpr (R % 4 == 0) {
 #pragma unroll
                 for (int q = 0; q < R / 4; ++q)
-                    lds128(src + 16 * q, dstw[row][4 * q], dstw[row][4 * q + 1], dstw[row][4 * q + 2],
-                           dstw[row][4 * q + 3]);
+                    lds128(src + 16 * q, cw[row][4 * q], cw[row][4 * q + 1], cw[row][4 * q + 2], cw[row][4 * q + 3]);
             } else if constexpr (R % 2 == 0) {
 #pragma unroll
-                for (int q = 0; q < R / 2; ++q) lds64(src + 8 * q, dstw[row][2 * q], dstw[row][2 * q + 1]);
+                for (int q = 0; q < R / 2; ++q) lds64(src + 8 * q, cw[row][2 * q], cw[row][2 * q + 1]);
             } else {
 #pragma unroll
-                for (int q = 0; q < R; ++q) lds32(src + 4 * q, dstw[row][q]);
+                for (int q = 0; q < R; ++q) lds32(src + 4 * q, cw[row][q]);
             }
         }
-        __syncwarp();                               // every lane's loads are ordered before ...
-        if (lane == 0) {
-            // ... the count (release); the last of the CTA's warps to count has all the others'
-            // loads behind it (acquire), resets the counter and refills the stage
-            if (atom_add_acq_rel_shared(cnt_u32 + slot * 4, 1u) == (uint32_t)kRingWarps - 1u) {
-                st_shared_u32(cnt_u32 + slot * 4, 0u);
-                if (c_left > (uint32_t)S) issue_unit(r_tile, r_w, slot);
-            }
-        }
-        if (++r_w == W) { r_w = 0; r_tile += gridDim.x; }
-        --c_left;
+        held_bar = c_bar;
         c_off += L::kUnitBytes;
-        if (c_off == (uint32_t)(S * L::kUnitBytes)) { c_off = 0; c_par ^= 1u; }
+        c_bar += 8;
+        if (c_bar == 8u * S) { c_off = 0; c_bar = 0; c_par ^= 1u; }
         return true;
     };
-    // the W terms of one worker for my 64 outputs: groups of FIT consecutive codes, one
-    // funnel shift brings a group's first field to bit 0, then every field lies below bit 23
-    uint64_t acc2[32];                          // output j of (row A, row B) as an fp32 pair
-    auto sum_unit = [&](const uint32_t (&cw)[2][R], const uint64_t a2) {
+    // `zero` is 0, but only at run time: (x & zero) makes the vote below depend on one word of
+    // every shared load of the unit in every lane, so the loads have completed when it is taken
+    // (a barrier among the lanes alone does not wait for loads in flight).
+    const uint32_t zero = *reinterpret_cast<volatile uint32_t*>(dsm + 264);
+    auto release_unit = [&]() {
+        constexpr int kStep = (R % 4 == 0) ? 4 : (R % 2 == 0) ? 2 : 1;    // words per load
+        uint32_t x = 0;
 #pragma unroll
-        for (int j0 = 0; j0 < 32; j0 += FIT) {
-            const int bit = j0 * R, wi = bit >> 5, sh = bit & 31;
-            uint32_t word[2];
+        for (int row = 0; row < 2; ++row)
 #pragma unroll
-            for (int row = 0; row < 2; ++row)
-                word[row] = (sh == 0) ? cw[row][wi]
-                          : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cw[row][wi] >> sh)
-                          : __funnelshift_r(cw[row][wi], cw[row][wi + 1], sh);
-            const uint64_t w2 = ((uint64_t)word[1] << 32) | word[0];
-#pragma unroll
-            for (int i = 0; i < FIT && j0 + i < 32; ++i) {
-                const uint64_t m2 = ((uint64_t)(mask << (i * R)) << 32) | (uint64_t)(mask << (i * R));
-                // (c - s) 2^(iR) a, rows A and B in one instruction
-                acc2[j0 + i] = fma2(sub2((w2 & m2) | magic2, T2[i]), a2, acc2[j0 + i]);
-            }
-        }
+            for (int q = 0; q < R; q += kStep) x ^= cw[row][q];
+        const bool done = __all_sync(0xFFFFFFFFu, (x & zero) == 0u);         // always true
+        if (done && lane == 0) mbar_arrive(bar_empty + held_bar);
     };
 
-    if (ok && n_units) ok = take_unit(cwa);
+    bool ok = true;
+    const float2* const a_mine = a_tab + grp;
 
     for (uint32_t ti = 0; ok && ti < my_tiles; ++ti) {
         const uint32_t tile = blockIdx.x + ti * gridDim.x;
@@ -267,20 +226,21 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         __syncwarp();
         if (ti + 1 < my_tiles) fetch_scales(tile + gridDim.x);
 
+        const uint32_t sub_a = tile * kRingSubs + warp, sub_b = sub_a + kRingWarps;
+        uint64_t acc2[32];                      // output j of (row A, row B) as an fp32 pair
 #pragma unroll
         for (int j = 0; j < 32; ++j) acc2[j] = 0ull;
         if (!first) {
             // running sums of the earlier messages (this path serves more than 64 messages
             // only): every lane reads its own two rows, 128 contiguous bytes each, and gives
             // the sums the powers of two of their fields
-            const uint32_t sub_a = tile * kRingSubs + warp, sub_b = sub_a + kRingWarps;
             const float4* src_a = reinterpret_cast<const float4*>(
                 dst.out + (uint64_t)sub_a * kDecTileElems + (uint32_t)lane * 32);
             const float4* src_b = reinterpret_cast<const float4*>(
                 dst.out + (uint64_t)sub_b * kDecTileElems + (uint32_t)lane * 32);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-                const float4 va = src_a[c];                     // sub_a < n_subs for every tile
+                const float4 va = sub_a < n_subs ? src_a[c] : make_float4(0.f, 0.f, 0.f, 0.f);
                 const float4 vb = sub_b < n_subs ? src_b[c] : make_float4(0.f, 0.f, 0.f, 0.f);
                 const float ia[4] = {va.x, va.y, va.z, va.w}, ib[4] = {vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
@@ -291,67 +251,130 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
             }
         }
 
-        const float2* const a_mine = a_tab + grp;
 #pragma unroll 1
         for (uint32_t w = 0; w < W; ++w) {
+            if (!take_unit()) { ok = false; break; }
             const uint64_t a2 = *reinterpret_cast<const uint64_t*>(a_mine + w);       // (a_A, a_B)
-            sum_unit(cwa, a2);
-            if (c_left) { if (!take_unit(cwa)) { ok = false; break; } }
+            // groups of FIT consecutive codes: one funnel shift brings a group's first field
+            // to bit 0, then every field lies below bit 23
+#pragma unroll
+            for (int j0 = 0; j0 < 32; j0 += FIT) {
+                const int bit = j0 * R, wi = bit >> 5, sh = bit & 31;
+                uint32_t word[2];
+#pragma unroll
+                for (int row = 0; row < 2; ++row)
+                    word[row] = (sh == 0) ? cw[row][wi]
+                              : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cw[row][wi] >> sh)
+                              : __funnelshift_r(cw[row][wi], cw[row][wi + 1 < R ? wi + 1 : wi], sh);
+                const uint64_t w2 = ((uint64_t)word[1] << 32) | word[0];
+#pragma unroll
+                for (int i = 0; i < FIT && j0 + i < 32; ++i) {
+                    const uint64_t m2 = ((uint64_t)(mask << (i * R)) << 32) | (uint64_t)(mask << (i * R));
+                    // (c - s) 2^(iR) a, rows A and B in one instruction
+                    acc2[j0 + i] = fma2(sub2((w2 & m2) | magic2, T2[i]), a2, acc2[j0 + i]);
+                }
+            }
+            release_unit();
         }
         if (!ok) break;
 
-        // undo the powers of two, divide by W; one row at a time through the staging buffer:
-        // row-per-lane -> coalesced 16-byte stores
+        // undo the powers of two, divide by W, store: 32 bytes (one sector) per store
 #pragma unroll
         for (int row = 0; row < 2; ++row) {
-            const uint32_t sub = tile * kRingSubs + warp + row * kRingWarps;
-            if (sub >= n_subs) break;
-            float acc[32];
+            const uint32_t sub = row ? sub_b : sub_a;
+            if (sub >= n_subs) continue;
+            const uint64_t o = (uint64_t)sub * kDecTileElems + (uint32_t)lane * 32;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float lo, hi;
-                unpack2(acc2[j], lo, hi);
-                acc[j] = row ? hi : lo;
+            for (int c = 0; c < 4; ++c) {
+                float v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int j = 8 * c + k;
+                    float lo, hi;
+                    unpack2(acc2[j], lo, hi);
+                    const float x = __fmul_rn(row ? hi : lo, __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23));
+                    v[k] = !last ? x : w_pow2 ? __fmul_rn(x, w_recip) : __fdiv_rn(x, w_total);
+                }
+                if (last) emit8(dst, o + 8 * c, v);
+                else stg256(dst.out + o + 8 * c, v);
             }
-            if (!last) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    acc[j] = __fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23));
-            } else if (w_pow2) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    acc[j] = __fmul_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), w_recip);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    acc[j] = __fdiv_rn(__fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23)), w_total);
-            }
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<float4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) =
-                    make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
-            __syncwarp();
-            const uint64_t o = (uint64_t)sub * kDecTileElems;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int idx = k * 32 + lane, rw = idx >> 3, ch = idx & 7;
-                const float4 v = *reinterpret_cast<const float4*>(stage + rw * 128 + ((ch ^ (rw & 7)) << 4));
-                if (last) emit4(dst, o + idx * 4, v);
-                else *reinterpret_cast<float4*>(dst.out + o + idx * 4) = v;
-            }
-            __syncwarp();
         }
     }
     cp_async_wait<0>();
-
-    // A wait ran out (a copy that never completed): flag it, and let the copies that were
-    // issued land before the CTA gives its shared memory back.
     if (!ok) { *s_abort = 1; if (lane == 0) atomicOr(status, kStatusTimeout); }
+}
+
+template <int R, bool CARRY>
+__global__ void __launch_bounds__(kRingThreads, 1)
+decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
+                   const DecodeOut dst, const uint32_t n_subs, const uint64_t n_words,
+                   const float w_recip, const int w_pow2, const uint32_t exp23_bits,
+                   const DecodeSlice sl, uint32_t* status) {
+    using L = DecodeRing<R>;
+    const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
+    const float w_total = CARRY ? sl.w_total : (float)W;
+    constexpr int S = L::kStages;
+    constexpr uint32_t mask = (1u << R) - 1u;
+    extern __shared__ __align__(128) uint8_t dsm[];
+    const uint32_t sm0 = smem_u32(dsm);
+    const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
+    volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 256);
+    volatile uint32_t* const s_issued = reinterpret_cast<volatile uint32_t*>(dsm + 260);   // units the producer issued
+    const int lane = threadIdx.x & 31;
+    // broadcast from lane 0 so that the compiler knows the value is warp-uniform
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
+
+    const uint32_t n_tiles = (n_subs + kRingSubs - 1) / kRingSubs;
+    const uint32_t my_tiles =
+        blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t n_units = my_tiles * W;                          // < 2^32: checked by the host
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, kRingWarps);
+        }
+        *s_abort = 0;
+        *s_issued = 0;
+        *reinterpret_cast<volatile uint32_t*>(dsm + 264) = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    if (warp == kRingWarps) {
+        // ---- producer: unit n = (my tile n / W, worker n % W), in order, into stage n % S ----
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t tile = blockIdx.x, w = 0, slot = 0, par = 0, u = 0;
+            for (; u < n_units; ++u) {
+                // stages are free the first time round; later the consumers hand them back
+                if (u >= (uint32_t)S && !mbar_wait(bar_empty + 8 * slot, par ^ 1u)) { ok = false; break; }
+                const uint32_t subs = min((uint32_t)kRingSubs, n_subs - tile * kRingSubs);
+                const uint32_t bytes = subs * (R * 128);
+                const uint32_t bar = bar_full + 8 * slot;
+                mbar_arrive_expect_tx(bar, bytes);
+                bulk_load_1d(sm0 + L::kRingOff + slot * L::kUnitBytes,
+                             tab.codes[w] + (uint64_t)tile * (R * 32 * kRingSubs), bytes, bar);
+                if (++w == W) { w = 0; tile += gridDim.x; }
+                if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; }
+            }
+            *s_issued = u;
+            if (!ok) { *s_abort = 1; atomicOr(status, kStatusTimeout); }    // a stage never came back
+        }
+        __syncwarp();
+    } else {
+        decode_ring_consumer<R, CARRY>(P, W, tab, dst, n_subs, w_recip, w_pow2, exp23_bits, first, last,
+                                       w_total, my_tiles, warp, lane, dsm, status);
+    }
     __syncthreads();
     if (*s_abort) {
-        if (threadIdx.x == 0)
-            for (int i = 0; i < S; ++i)
-                if (s_issued[i]) mbar_wait(bar_full + 8 * i, (s_issued[i] - 1u) & 1u);
+        // a wait ran out: let the copies in flight land before the CTA gives its shared memory
+        // back (unit v went into stage v % S; the last S units may still be on their way)
+        if (threadIdx.x == 0) {
+            const uint32_t u = *s_issued;
+            for (uint32_t v = (u > (uint32_t)S ? u - S : 0); v < u; ++v)
+                mbar_wait(bar_full + 8 * (v % S), (v / S) & 1u);
+        }
         return;
     }
 
