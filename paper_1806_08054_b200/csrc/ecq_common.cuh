@@ -135,7 +135,7 @@ __device__ __forceinline__ void fence_mbar_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 
-// 2-D tiled TMA load into this CTA's shared memory (no multicast).
+// 2-D tiled TMA load into this CTA's own shared memory.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y,
                                             uint32_t bar) {
     asm volatile(
