@@ -306,6 +306,11 @@ encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
             m = __float_as_uint(ss);
         }
         if (rpb > 32 && lane == 0) s_wmax[warp] = m;
+        // The barrier below hands the load buffer to the next tile's copy, so every thread's
+        // shared loads of G and H must have completed by then, which the barrier itself does not
+        // wait for.  m depends on all of them, and the shuffles above consume it; with one row
+        // per bucket there is no shuffle, so one is made here (it returns m).
+        if (rpb == 1) m = __shfl_sync(0xFFFFFFFFu, m, lane);
         __syncthreads();                                   // the load buffer is free
         if (*s_abort) break;                               // uniform: set before the barrier
         if (tid == 0 && T + gridDim.x < total_tiles) issue_load(T + gridDim.x);
