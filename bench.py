@@ -43,7 +43,7 @@ NOMINAL_HBM_GBS = 8000.0
 # over 11,310,497,792 entries; see profiles/encode_tiled_kernel.md), keyed by (bucket, levels).
 # Traffic grows in proportion to the entries of a launch.  Set an entry to None when the
 # kernel changes.
-NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): 141431158016 / 11310497792}
+NCU_DRAM_BYTES_PER_ENTRY = {(512, 4): 141431376025 / 11310497792}
 
 
 def code_bits(s: int) -> int:
