@@ -251,7 +251,9 @@ __device__ __forceinline__ void decode_ring_consumer(
             }
         }
 
-#pragma unroll 1
+        // (four workers per loop turn: 7 % fewer instructions than one per turn; the words are
+        // still loaded at the top of each worker's part)
+#pragma unroll 4
         for (uint32_t w = 0; w < W; ++w) {
             if (!take_unit()) { ok = false; break; }
             const uint64_t a2 = *reinterpret_cast<const uint64_t*>(a_mine + w);       // (a_A, a_B)
