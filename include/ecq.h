@@ -14,7 +14,7 @@
  *     is the default stream) and the call returns without synchronising,
  *     unless stated otherwise.
  *   - `grad`, `err`, `out`, `codes` must be 16-byte aligned; `scales` 4-byte.
- *   - A context is immutable after creation (except ecq_set_error_mode, ecq_set_norm and ecq_set_decode_plan) and may
+ *   - A context is immutable after creation (except the ecq_set_* calls) and may
  *     be used from several host threads on different streams.
  *   - Inputs must be finite.  A bucket whose compensated values contain NaN or
  *     Inf is sent as all-zero levels with scale 0, its accumulator entries are
@@ -66,8 +66,9 @@ enum {
  *   beta    time-decay factor of Eq. 5/6 (0 <= beta <= 1)
  *   seed    64-bit key of the Philox4x32-10 stream that drives Eq. 9
  * The context owns only constants and one 4-byte device status word on the
- * device that is current at the time of the call.  ECQ_ERR_ARG on a range
- * violation, ECQ_ERR_ALLOC / ECQ_ERR_CUDA otherwise.
+ * device that is current at the time of the call (device ordinals 0..63; beyond
+ * that ECQ_ERR_CUDA).  ECQ_ERR_ARG on a range violation, ECQ_ERR_ALLOC /
+ * ECQ_ERR_CUDA otherwise.
  */
 int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels,
                float alpha, float beta, uint64_t seed);
@@ -84,8 +85,8 @@ void ecq_destroy(ecq_ctx* ctx);
 int ecq_set_error_mode(ecq_ctx* ctx, int mode);
 
 /*
- * Choose the scaling factor ||v|| of Eq. 8 ("possible choices include l2-norm and
- * l-infinity-norm"), taken per bucket.
+ * Choose the scaling factor ||v|| of Eq. 8 (the paper leaves the norm open and names l2 and
+ * l-infinity), taken per bucket.
  *   0 (default)  l-infinity: max |v_i|
  *   1            l2: sqrt(sum v_i^2).  The fp32 sum has a fixed order so that results do not
  *                depend on the kernel's shape: every run of 32 consecutive entries is summed
@@ -116,6 +117,20 @@ int ecq_set_norm(ecq_ctx* ctx, int norm);
 #define ECQ_DECODE_WARP 1
 #define ECQ_DECODE_RING 2
 int ecq_set_decode_plan(ecq_ctx* ctx, int kernel, uint32_t max_ctas);
+
+/*
+ * Set how many times a kernel polls for an asynchronous copy (a TMA or bulk load into
+ * shared memory) before it gives up.  The paper has no counterpart: this is the library's
+ * guard against a copy that never completes.  A wait that runs out makes its CTA stop,
+ * records ECQ_ERR_TIMEOUT in the sticky status word (ecq_status), lets the copies still in
+ * flight land -- that last wait always keeps the built-in limit of 2^22 polls, whatever is
+ * set here -- and returns; buffers the CTA had not finished are left partly written, and
+ * the context stays usable.  Default 2^22 (a fraction of a second; no copy takes that
+ * long).  0 makes every wait give up at once without polling: the only use of small
+ * values is to exercise that path.
+ */
+#define ECQ_WAIT_LIMIT_DEFAULT (1u << 22)
+int ecq_set_wait_limit(ecq_ctx* ctx, uint32_t polls);
 
 /* r = ceil(log2(2s+1)): bits per entry (paragraph after Eq. 9). */
 uint32_t ecq_code_bits(const ecq_ctx* ctx);
@@ -314,9 +329,12 @@ int ecq_step_host(ecq_ctx* ctx, uint32_t W, uint32_t step,
  *
  * The call enqueues on `cuda_stream`, waits for it, and returns ECQ_OK,
  * ECQ_ERR_NONFINITE or ECQ_ERR_TIMEOUT like ecq_status would.  It calls no
- * cudaMalloc / cudaFree and no allocating library routine.  The first call on a
- * device looks up the scratch array's device address (with that device current);
- * make that first call outside any stream capture.  All calls on a device share
+ * cudaMalloc / cudaFree and no allocating library routine (a host thread's first
+ * call binds the device's primary context with cudaSetDevice; kernels are loaded
+ * by the CUDA runtime on first use as for any library).  The first call on a
+ * device (ordinals 0..63; beyond that ECQ_ERR_CUDA) looks up the scratch array's
+ * device address (with that device current); make that first call outside any
+ * stream capture.  All calls on a device share
  * the one array and it keeps the last call's contents: the status word is cleared
  * at the start of every call, the messages are fully overwritten; two calls that
  * overlap on the GPU (different streams or host threads) race on it and must be

@@ -24,6 +24,7 @@ ECQ_HUFFMAN_CHUNK = 1024
 ECQ_HUFFMAN_TABLE_BYTES = 4096 * 4 + 4096 * 4 + 16
 ECQ_STATIC_SCRATCH_BYTES = 4 << 20
 ECQ_MAX_WORKERS = 64
+ECQ_WAIT_LIMIT_DEFAULT = 1 << 22
 ECQ_MAX_WORKERS_TOTAL = 1024
 
 _lib = None
@@ -56,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.ecq_set_norm.restype = i32
         L.ecq_set_decode_plan.argtypes = [vp, i32, ctypes.c_uint32]
         L.ecq_set_decode_plan.restype = i32
+        L.ecq_set_wait_limit.argtypes = [vp, ctypes.c_uint32]
+        L.ecq_set_wait_limit.restype = i32
         L.ecq_code_bits.argtypes = [vp]
         L.ecq_code_bits.restype = u32
         L.ecq_num_buckets.argtypes = [vp]
@@ -154,6 +157,13 @@ def ecq_set_decode_plan(ctx: int, kernel: int = ECQ_DECODE_AUTO, max_ctas: int =
     rc = lib().ecq_set_decode_plan(ctx, kernel, max_ctas)
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_set_decode_plan")
+
+
+def ecq_set_wait_limit(ctx: int, polls: int) -> None:
+    """Polls an in-kernel wait for an asynchronous copy makes before it gives up (default 2**22)."""
+    rc = lib().ecq_set_wait_limit(ctx, polls)
+    if rc != ECQ_OK:
+        raise EcqError(rc, "ecq_set_wait_limit")
 
 
 def ecq_code_bits(ctx: int) -> int:
@@ -264,6 +274,8 @@ def ecq_step_static(d: int, bucket: int, levels: int, alpha: float, beta: float,
     the device status (ECQ_OK / ECQ_ERR_NONFINITE / ECQ_ERR_TIMEOUT) and raises on argument
     errors, among them ECQ_ERR_TOO_LARGE when the messages exceed the built-in scratch."""
     W = len(grads)
+    if any(g.numel() < d for g in grads) or err.numel() < W * d or out.numel() < d:
+        raise ValueError("ecq_step_static: grads need d entries each, err W*d, out d")
     gp = (ctypes.c_void_p * W)(*[_dev(g, torch.float32, "grads") for g in grads])
     rc = lib().ecq_step_static(d, bucket, levels, alpha, beta, seed, W, step, gp,
                                _dev(err, torch.float32, "err"), _dev(out, torch.float32, "out"),

@@ -45,6 +45,10 @@ EncodeTiledFn tensor_map_encoder() {
     return fn;
 }
 
+// Per-device set-up (kernel attributes, the built-in scratch's address) is kept in tables
+// indexed by the device ordinal; contexts on devices beyond them are refused.
+constexpr int kMaxDevices = 64;
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
@@ -60,6 +64,7 @@ struct ecq_ctx {
     bool tiled_ok;               // bucket is a power of two <= 4096
     int decode_kernel;           // ECQ_DECODE_AUTO / _WARP / _RING (ecq_set_decode_plan)
     uint32_t decode_max_ctas;    // 0: fill the device
+    uint32_t wait_limit;         // polls an in-kernel wait makes before it gives up
     // lazily created by ecq_step_host
     std::mutex host_mu;
     cudaStream_t copy_stream;
@@ -84,8 +89,13 @@ bool make_tile_map(CUtensorMap* tm, const float* base, uint64_t rows, uint32_t b
     if (!enc) return false;
     // the encoder is a driver call: a host thread that has made no runtime call yet has no
     // context bound, so bind the current device's primary context once per thread
+    // (cudaSetDevice does that and allocates nothing)
     thread_local bool context_bound = false;
-    if (!context_bound) { cudaFree(nullptr); context_bound = true; }
+    if (!context_bound) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaSetDevice(dev) != cudaSuccess) return false;
+        context_bound = true;
+    }
     const cuuint64_t dims[2] = {32, rows};
     const cuuint64_t strides[1] = {128};
     const cuuint32_t box[2] = {32, box_rows};
@@ -110,9 +120,9 @@ template <int R, bool MODE1, int ROWS>
 int launch_encode_tiled(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, uint32_t step,
                         const WorkerBuffers* wb, cudaStream_t st, uint32_t n_tiles) {
     using L = EncodeSmem<R, ROWS>;
-    static std::once_flag once[16];
-    static int occ[16];
-    const int dev = c->device & 15;
+    static std::once_flag once[kMaxDevices];
+    static int occ[kMaxDevices];
+    const int dev = c->device;                            // < kMaxDevices: checked at creation
     auto kern = encode_tiled_kernel<R, MODE1, ROWS>;
     std::call_once(once[dev], [&] {
         int o = 0;
@@ -140,7 +150,8 @@ int launch_encode_tiled(ecq_ctx* c, uint32_t worker_base, uint32_t n_workers, ui
     const uint64_t total = (uint64_t)n_tiles * n_workers;
     uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
     if (grid > total) grid = (uint32_t)total;
-    kern<<<grid, ROWS, L::kTotal, st>>>(bt, c->P, worker_base, n_workers, step, c->d_status, n_tiles);
+    kern<<<grid, ROWS, L::kTotal, st>>>(bt, c->P, worker_base, n_workers, step, c->d_status, n_tiles,
+                                        c->wait_limit);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? ECQ_OK : ECQ_ERR_CUDA;
 }
@@ -232,9 +243,9 @@ bool launch_decode_tiled(ecq_ctx* c, uint32_t W, const MessageTable& tab, Decode
     const uint32_t gsz = B >= 1024 ? 32 : B / 32;
     if (W > (uint32_t)kDecAreg * gsz) return false;
     if (n_tiles64 * W > 0xFFFFFFFFull) return false;
-    static std::once_flag once[16];
-    static int occ[16];
-    const int dev = c->device & 15;
+    static std::once_flag once[kMaxDevices];
+    static int occ[kMaxDevices];
+    const int dev = c->device;                            // < kMaxDevices: checked at creation
     auto kern = decode_tiled_kernel<R, CARRY>;
     std::call_once(once[dev], [&] {
         int o = 0;
@@ -271,9 +282,9 @@ bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeO
         return false;
     const uint64_t n_tiles = (n_subs64 + kRingSubs - 1) / kRingSubs;
     if (n_tiles * W > 0xFFFFFFFFull) return false;
-    static std::once_flag once[16];
-    static int occ[16];
-    const int dev = c->device & 15;
+    static std::once_flag once[kMaxDevices];
+    static int occ[kMaxDevices];
+    const int dev = c->device;                            // < kMaxDevices: checked at creation
     auto kern = decode_ring_kernel<R, CARRY>;
     std::call_once(once[dev], [&] {
         int o = 0;
@@ -291,7 +302,8 @@ bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeO
     if (c->decode_max_ctas && grid > c->decode_max_ctas) grid = c->decode_max_ctas;
     if (grid > n_tiles) grid = (uint32_t)n_tiles;
     kern<<<grid, kRingThreads, L::kSmem, st>>>(c->P, W, tab, out, (uint32_t)n_subs64, c->n_words,
-                                                  w_recip, w_pow2, 0x4B000000u, sl, c->d_status);
+                                                  w_recip, w_pow2, L::kHalf ? 0x64006400u : 0x4B000000u,
+                                                  c->wait_limit, sl, c->d_status);
     return true;
 }
 
@@ -389,9 +401,10 @@ int ecq_create(ecq_ctx** out, uint64_t d, uint32_t bucket, uint32_t levels, floa
     c->tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= kMaxTiledBucket;
     c->decode_kernel = ECQ_DECODE_AUTO;
     c->decode_max_ctas = 0;
+    c->wait_limit = kWaitLimit;
     c->host_ready = false;
     c->d_status = nullptr; c->h_status = nullptr;
-    if (cudaGetDevice(&c->device) != cudaSuccess ||
+    if (cudaGetDevice(&c->device) != cudaSuccess || c->device < 0 || c->device >= kMaxDevices ||
         cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
         delete c; return ECQ_ERR_CUDA;
     }
@@ -429,6 +442,12 @@ int ecq_set_decode_plan(ecq_ctx* c, int kernel, uint32_t max_ctas) {
     if (!c || kernel < ECQ_DECODE_AUTO || kernel > ECQ_DECODE_RING) return ECQ_ERR_ARG;
     c->decode_kernel = kernel;
     c->decode_max_ctas = max_ctas;
+    return ECQ_OK;
+}
+
+int ecq_set_wait_limit(ecq_ctx* c, uint32_t polls) {
+    if (!c) return ECQ_ERR_ARG;
+    c->wait_limit = polls;
     return ECQ_OK;
 }
 
@@ -808,11 +827,11 @@ struct StaticScratch {
     unsigned char* ptr = nullptr;
     cudaError_t err = cudaErrorUnknown;
 };
-StaticScratch g_static[16];
+StaticScratch g_static[kMaxDevices];
 
 // Device address of the built-in scratch on the current device (set-up on first use).
 unsigned char* static_scratch_ptr(int device) {
-    StaticScratch& s = g_static[device & 15];
+    StaticScratch& s = g_static[device];                  // < kMaxDevices: checked by the caller
     std::call_once(s.once, [&] {
         void* p = nullptr;
         s.err = cudaGetSymbolAddress(&p, g_static_scratch);
@@ -853,6 +872,7 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
     c.tiled_ok = (bucket & (bucket - 1)) == 0 && bucket <= kMaxTiledBucket;
     c.decode_kernel = ECQ_DECODE_AUTO;
     c.decode_max_ctas = 0;
+    c.wait_limit = kWaitLimit;
     c.host_ready = false;
     c.h_status = nullptr;
 
@@ -861,7 +881,7 @@ extern "C" int ecq_step_static(uint64_t d, uint32_t bucket, uint32_t levels, flo
     const uint64_t need = 256 + (uint64_t)W * (codes_b + scales_b);
     if (need > ECQ_STATIC_SCRATCH_BYTES) return ECQ_ERR_TOO_LARGE;
 
-    if (cudaGetDevice(&c.device) != cudaSuccess ||
+    if (cudaGetDevice(&c.device) != cudaSuccess || c.device < 0 || c.device >= kMaxDevices ||
         cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess)
         return ECQ_ERR_CUDA;
     unsigned char* scratch = static_scratch_ptr(c.device);

@@ -1,5 +1,5 @@
 // Receiver-side kernel for long vectors: unpack -> dequantise -> W-way mean (Eq. 4;
-// Algorithm 1, "compute global gradients"), with the code words brought in by bulk copies
+// Algorithm 1, phase 2, global-gradient step), with the code words brought in by bulk copies
 // that a whole CTA shares.
 //
 // One CTA per SM: 15 consumer warps and one producer warp.  A CTA tile is 30 sub-tiles of
@@ -10,11 +10,19 @@
 //     mbarrier.  Lane 0 of the producer warp issues the copies in order, each as soon as
 //     the 15 consumer warps have handed its stage back on the "empty" mbarrier.  Per unit a
 //     consumer warp spends a wait, two shared loads and an arrive on data movement;
-//   * the two rows of a lane travel as the two halves of packed fp32x2 registers:
-//     (word_A & field, word_B & field) | 2^23 exponent bits is (2^23 + c 2^p) for both rows,
-//     one packed subtract leaves ((c - s) 2^p), one packed multiply-add with the pair of
-//     level steps (a_A, a_B) of the rows' buckets adds the terms; per worker the chain
-//     acc <- fma(q_w, a_w, acc) is the one Eq. 4 writes out, in ascending w;
+//   * the two rows of a lane travel as the two halves of packed fp32x2 registers: one packed
+//     multiply-add with the pair of level steps (a_A, a_B) of the rows' buckets adds the
+//     terms; per worker the chain acc <- fma(q_w, a_w, acc) is the one Eq. 4 writes out, in
+//     ascending w;
+//   * turning a bit field into the float q = c - s is what the kernel is bound by: issue
+//     slots (a packed fp32x2 instruction takes two, so packing saves none) and the 16-lane
+//     logic pipe.  For code widths that divide 16 the fields are merged two at a time into
+//     an fp16 pair: (word & field-in-both-halves) | 0x64006400 is (1024 + c 2^p) twice, and
+//     one mixed-precision add per code (f16 + f32 -> f32) takes 1024 + s 2^p off and widens,
+//     exactly: half a logic instruction and one add per code.  Other widths merge the field
+//     into the mantissa of 2^23, (word_A & field, word_B & field) | 2^23 bits, and one packed
+//     subtract leaves ((c - s) 2^p) for both rows: one logic instruction and half a packed
+//     subtract (one slot) per code;
 //   * level steps a_w = scale_w / s of the next tile are fetched with 4-byte asynchronous
 //     copies while this tile is summed;
 //   * a lane stores its rows with 32-byte stores (whole sectors), so the means need no
@@ -38,6 +46,12 @@ constexpr int kRingMinTilesPerCta = 12;
 constexpr int kRingMaxAutoBits = 8;
 
 template <int R> struct DecodeRing {
+    static constexpr bool kHalf = (R == 2 || R == 4 || R == 8);
+    static constexpr int kHalfFields = 16 / R;
+    static constexpr int kViewFields = 10 / R;
+    __host__ __device__ static constexpr int field_shift(int j) {
+        return kHalf ? (((j % (32 / R)) % kHalfFields) % kViewFields) * R : (j % (R == 2 ? 8 : R == 3 ? 7 : R == 4 ? 4 : 23 / R)) * R;
+    }
     static constexpr int kUnitBytes = R * 128 * kRingSubs;
     // whole fields below bit 23 of a word; chosen so that the fewest groups need a shift
     static constexpr int kFit = R == 2 ? 8 : R == 3 ? 7 : R == 4 ? 4 : 23 / R;
@@ -91,6 +105,13 @@ __device__ __forceinline__ void emit8(const DecodeOut& o, uint64_t i, const floa
     }
     if (o.out) stg256(o.out + i, v);
 }
+__device__ __forceinline__ void add_f32_f16x2(uint32_t m, float c, float& lo, float& hi) {
+    asm("{\n\t.reg .b16 h0, h1;\n\t"
+        "mov.b32 {h0, h1}, %2;\n\t"
+        "add.rn.f32.f16 %0, h0, %3;\n\t"
+        "add.rn.f32.f16 %1, h1, %3;\n\t}"
+        : "=f"(lo), "=f"(hi) : "r"(m), "f"(c));
+}
 __device__ __forceinline__ void lds32(uint32_t a, uint32_t& x) {
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x) : "r"(a) : "memory");
 }
@@ -107,7 +128,7 @@ __device__ __forceinline__ void decode_ring_consumer(
         const CodecParams& P, const uint32_t W, const MessageTable& tab, const DecodeOut& dst,
         const uint32_t n_subs, const float w_recip, const int w_pow2, const uint32_t exp23_bits,
         const bool first, const bool last, const float w_total, const uint32_t my_tiles,
-        const int warp, const int lane, uint8_t* dsm, uint32_t* status) {
+        const uint32_t wait_limit, const int warp, const int lane, uint8_t* dsm, uint32_t* status) {
     using L = DecodeRing<R>;
     constexpr int S = L::kStages;
     constexpr int FIT = L::kFit;
@@ -138,6 +159,9 @@ __device__ __forceinline__ void decode_ring_consumer(
     // the exponent bits arrive as a kernel argument so that they live in a register: a
     // logic instruction takes one immediate, and the field mask is it
     const uint64_t magic2 = ((uint64_t)exp23_bits << 32) | exp23_bits;
+    float subh[L::kViewFields > 0 ? L::kViewFields : 1];
+#pragma unroll
+    for (int i = 0; i < L::kViewFields; ++i) subh[i] = -__fmaf_rn(P.sf, (float)(1u << (i * R)), 1024.f);
 
     // ---- raw scales of a tile's buckets: worker k*gsz + gl of my group, rows A and B ----
     auto fetch_scales = [&](uint32_t tile) {
@@ -168,7 +192,7 @@ __device__ __forceinline__ void decode_ring_consumer(
     // top of every turn keeps the words out of the loop-carried state (carrying them from the
     // end of the previous turn cost 20 register moves a unit).
     auto take_unit = [&]() -> bool {
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_full + c_bar, c_par))) return false;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_n(bar_full + c_bar, c_par, wait_limit))) return false;
 #pragma unroll
         for (int row = 0; row < 2; ++row) {
             const uint32_t src = my_off + c_off + row * (kRingWarps * R * 128);
@@ -245,7 +269,7 @@ __device__ __forceinline__ void decode_ring_consumer(
                 const float ia[4] = {va.x, va.y, va.z, va.w}, ib[4] = {vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const float e = __uint_as_float((uint32_t)(127 - 22 + ((4 * c + q) % FIT) * R) << 23);
+                    const float e = __uint_as_float((uint32_t)(127 - 22 + L::field_shift(4 * c + q)) << 23);
                     acc2[4 * c + q] = pack2(__fmul_rn(ia[q], e), __fmul_rn(ib[q], e));
                 }
             }
@@ -257,6 +281,28 @@ __device__ __forceinline__ void decode_ring_consumer(
         for (uint32_t w = 0; w < W; ++w) {
             if (!take_unit()) { ok = false; break; }
             const uint64_t a2 = *reinterpret_cast<const uint64_t*>(a_mine + w);       // (a_A, a_B)
+            if constexpr (L::kHalf) {
+                constexpr int CW = 32 / R, NF = L::kHalfFields, FV = L::kViewFields;
+#pragma unroll
+                for (int wi = 0; wi < R; ++wi) {
+#pragma unroll
+                    for (int v0 = 0; v0 < NF; v0 += FV) {
+                        const uint32_t xa = v0 == 0 ? cw[0][wi] : (cw[0][wi] >> (v0 * R));
+                        const uint32_t xb = v0 == 0 ? cw[1][wi] : (cw[1][wi] >> (v0 * R));
+#pragma unroll
+                        for (int i = 0; i < FV && v0 + i < NF; ++i) {
+                            const uint32_t ma = (xa & ((mask << (i * R)) * 0x00010001u)) | exp23_bits;
+                            const uint32_t mb = (xb & ((mask << (i * R)) * 0x00010001u)) | exp23_bits;
+                            float la, ha, lb, hb;
+                            add_f32_f16x2(ma, subh[i], la, ha);
+                            add_f32_f16x2(mb, subh[i], lb, hb);
+                            const int jl = wi * CW + v0 + i, jh = jl + NF;
+                            acc2[jl] = fma2(pack2(la, lb), a2, acc2[jl]);
+                            acc2[jh] = fma2(pack2(ha, hb), a2, acc2[jh]);
+                        }
+                    }
+                }
+            } else {
             // groups of FIT consecutive codes: one funnel shift brings a group's first field
             // to bit 0, then every field lies below bit 23
 #pragma unroll
@@ -276,6 +322,7 @@ __device__ __forceinline__ void decode_ring_consumer(
                     acc2[j0 + i] = fma2(sub2((w2 & m2) | magic2, T2[i]), a2, acc2[j0 + i]);
                 }
             }
+            }
             release_unit();
         }
         if (!ok) break;
@@ -294,7 +341,7 @@ __device__ __forceinline__ void decode_ring_consumer(
                     const int j = 8 * c + k;
                     float lo, hi;
                     unpack2(acc2[j], lo, hi);
-                    const float x = __fmul_rn(row ? hi : lo, __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23));
+                    const float x = __fmul_rn(row ? hi : lo, __uint_as_float((uint32_t)(127 + 22 - L::field_shift(j)) << 23));
                     v[k] = !last ? x : w_pow2 ? __fmul_rn(x, w_recip) : __fdiv_rn(x, w_total);
                 }
                 if (last) emit8(dst, o + 8 * c, v);
@@ -311,7 +358,7 @@ __global__ void __launch_bounds__(kRingThreads, 1)
 decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
                    const DecodeOut dst, const uint32_t n_subs, const uint64_t n_words,
                    const float w_recip, const int w_pow2, const uint32_t exp23_bits,
-                   const DecodeSlice sl, uint32_t* status) {
+                   const uint32_t wait_limit, const DecodeSlice sl, uint32_t* status) {
     using L = DecodeRing<R>;
     const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
     const float w_total = CARRY ? sl.w_total : (float)W;
@@ -350,7 +397,8 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
             uint32_t tile = blockIdx.x, w = 0, slot = 0, par = 0, u = 0;
             for (; u < n_units; ++u) {
                 // stages are free the first time round; later the consumers hand them back
-                if (u >= (uint32_t)S && !mbar_wait(bar_empty + 8 * slot, par ^ 1u)) { ok = false; break; }
+                if (u >= (uint32_t)S && !mbar_wait_n(bar_empty + 8 * slot, par ^ 1u, wait_limit)) { ok = false; break; }
+                if (*s_abort) break;                        // a consumer's wait ran out
                 const uint32_t subs = min((uint32_t)kRingSubs, n_subs - tile * kRingSubs);
                 const uint32_t bytes = subs * (R * 128);
                 const uint32_t bar = bar_full + 8 * slot;
@@ -366,12 +414,13 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         __syncwarp();
     } else {
         decode_ring_consumer<R, CARRY>(P, W, tab, dst, n_subs, w_recip, w_pow2, exp23_bits, first, last,
-                                       w_total, my_tiles, warp, lane, dsm, status);
+                                       w_total, my_tiles, wait_limit, warp, lane, dsm, status);
     }
     __syncthreads();
     if (*s_abort) {
         // a wait ran out: let the copies in flight land before the CTA gives its shared memory
-        // back (unit v went into stage v % S; the last S units may still be on their way)
+        // back (unit v went into stage v % S; the last S units may still be on their way).
+        // This wait keeps the full limit whatever the context's.
         if (threadIdx.x == 0) {
             const uint32_t u = *s_issued;
             for (uint32_t v = (u > (uint32_t)S ? u - S : 0); v < u; ++v)

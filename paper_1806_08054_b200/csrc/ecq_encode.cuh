@@ -217,7 +217,7 @@ template <int R, bool MODE1, int ROWS>
 __global__ void __launch_bounds__(EncodeTile<ROWS>::kThreads, EncodeTile<ROWS>::kCtasPerSm)
 encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
                     const uint32_t worker_base, const uint32_t n_workers, const uint32_t step,
-                    uint32_t* status, const uint32_t n_tiles) {
+                    uint32_t* status, const uint32_t n_tiles, const uint32_t wait_limit) {
     using L = EncodeSmem<R, ROWS>;
     constexpr int kTileRows = ROWS, kTileElems = EncodeTile<ROWS>::kElems;
     constexpr int kTileBytes = EncodeTile<ROWS>::kBytes, kEncodeThreads = ROWS;
@@ -262,7 +262,7 @@ encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
     for (uint32_t T = blockIdx.x; T < total_tiles; T += gridDim.x, parity ^= 1u) {
         const uint32_t entry = T / n_tiles, tile = T - entry * n_tiles;
         const uint32_t worker = worker_base + entry;
-        if (!mbar_wait(bar_full, parity)) { *s_abort = 1; atomicOr(status, kStatusTimeout); }
+        if (!mbar_wait_n(bar_full, parity, wait_limit)) { *s_abort = 1; atomicOr(status, kStatusTimeout); }
 
         // my row of g and h -> registers
         float4 G[8], H[8];

@@ -41,14 +41,21 @@ def test_static_step_matches_the_ordinary_entry_points(d, bucket, levels, W):
     out_ref = torch.zeros(d, device="cuda")
     err = torch.zeros(W * d, device="cuda")
     out = torch.full((d,), -3.0, device="cuda")
-    for t in range(2):                                  # two calls in a row share the scratch
+    for t in range(3):                                  # calls in a row share the scratch
         grads = [_grad(d, w, t) for w in range(W)]
         for w in range(W):
             ecq.ecq_encode(ctx, w, t, grads[w], err_ref[w], codes[w], scales[w])
         ecq.ecq_decode_mean(ctx, codes, scales, out_ref)
         assert ecq.ecq_status(ctx) == ecq.ECQ_OK
+        torch.cuda.synchronize()
+        free_before, launches_before = torch.cuda.mem_get_info()[0], ecq.ecq_launch_count()
         rc = ecq.ecq_step_static(d, bucket, levels, alpha, beta, seed, t, grads, err, out)
         assert rc == ecq.ECQ_OK
+        assert ecq.ecq_launch_count() - launches_before == W + 1
+        if t > 0:
+            # what the entry point is for: once the kernels are loaded (first call), a call
+            # leaves the device's free memory exactly where it found it
+            assert torch.cuda.mem_get_info()[0] == free_before
         a, b = out.cpu().numpy(), out_ref.cpu().numpy()
         assert np.all(np.abs(a - b) <= 1e-7 + 1e-6 * np.abs(b))
         assert torch.equal(out, out_ref)
@@ -66,6 +73,20 @@ def test_static_step_reports_nonfinite_then_clears():
     assert ecq.ecq_step_static(d, 512, 4, 1.0, 0.9, 1, 0, grads, err, out) == ecq.ECQ_ERR_NONFINITE
     grads[1][17] = 0.0
     assert ecq.ecq_step_static(d, 512, 4, 1.0, 0.9, 1, 1, grads, err, out) == ecq.ECQ_OK
+
+
+def test_binding_checks_buffer_lengths():
+    d, W = 4096, 2
+    g = [torch.zeros(d, device="cuda") for _ in range(W)]
+    with pytest.raises(ValueError):
+        ecq.ecq_step_static(d, 512, 4, 1.0, 0.9, 1, 0, g, torch.zeros(W * d - 1, device="cuda"),
+                            torch.zeros(d, device="cuda"))
+    with pytest.raises(ValueError):
+        ecq.ecq_step_static(d, 512, 4, 1.0, 0.9, 1, 0, g, torch.zeros(W * d, device="cuda"),
+                            torch.zeros(d - 1, device="cuda"))
+    with pytest.raises(ValueError):
+        ecq.ecq_step_static(d, 512, 4, 1.0, 0.9, 1, 0, [g[0], g[1][:100]],
+                            torch.zeros(W * d, device="cuda"), torch.zeros(d, device="cuda"))
 
 
 def test_static_step_refuses_what_does_not_fit():
