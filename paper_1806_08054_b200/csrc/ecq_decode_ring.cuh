@@ -5,11 +5,12 @@
 // One CTA per SM: 15 consumer warps and one producer warp.  A CTA tile is 30 sub-tiles of
 // 1024 outputs.  Consumer warp k owns sub-tiles k and k + 15; a lane owns one run of 32
 // consecutive outputs ("row") in each, whose codes are R whole words.
-//   * unit (tile, worker) = the worker's code words of the tile, R * 3840 contiguous
-//     bytes: ONE bulk copy into a ring of stages, signalled on the stage's "full"
-//     mbarrier.  Lane 0 of the producer warp issues the copies in order, each as soon as
-//     the 15 consumer warps have handed its stage back on the "empty" mbarrier.  Per unit a
-//     consumer warp spends a wait, two shared loads and an arrive on data movement;
+//   * a ring stage holds the code words of (tile, kGroup consecutive workers): one bulk copy
+//     of R * 3840 contiguous bytes per worker, all counted on the stage's "full" mbarrier.
+//     Lane 0 of the producer warp issues them in order, each stage as soon as the 15 consumer
+//     warps have handed it back on its "empty" mbarrier.  A consumer warp waits once per
+//     stage, reads the stage's words of its two rows into registers (all loads first, so the
+//     shared-memory latency is met once), sums, and arrives once;
 //   * the two rows of a lane travel as the two halves of packed fp32x2 registers: one packed
 //     multiply-add with the pair of level steps (a_A, a_B) of the rows' buckets adds the
 //     terms; per worker the chain acc <- fma(q_w, a_w, acc) is the one Eq. 4 writes out, in
@@ -46,25 +47,29 @@ constexpr int kRingMinTilesPerCta = 12;
 constexpr int kRingMaxAutoBits = 8;
 
 template <int R> struct DecodeRing {
+    // fp16 pair merge where two fields sit 16 bits apart in a word
     static constexpr bool kHalf = (R == 2 || R == 4 || R == 8);
-    static constexpr int kHalfFields = 16 / R;
-    static constexpr int kViewFields = 10 / R;
-    __host__ __device__ static constexpr int field_shift(int j) {
-        return kHalf ? (((j % (32 / R)) % kHalfFields) % kViewFields) * R : (j % (R == 2 ? 8 : R == 3 ? 7 : R == 4 ? 4 : 23 / R)) * R;
-    }
-    static constexpr int kUnitBytes = R * 128 * kRingSubs;
-    // whole fields below bit 23 of a word; chosen so that the fewest groups need a shift
+    static constexpr int kHalfFields = 16 / R;                   // fields of a 16-bit half
+    static constexpr int kViewFields = 10 / R;                   // of which lie below bit 10 at a time
+    // fp32 merge: whole fields below bit 23 of a word; chosen so that the fewest groups need a shift
     static constexpr int kFit = R == 2 ? 8 : R == 3 ? 7 : R == 4 ? 4 : 23 / R;
-    // full mbarriers at 0, empty ones at 128, abort flag at 256, units issued at 260
+    // bit position of code j's field in the register it is merged from
+    __host__ __device__ static constexpr int field_shift(int j) {
+        return kHalf ? (((j % (32 / R)) % kHalfFields) % kViewFields) * R : (j % kFit) * R;
+    }
+    static constexpr int kGroup = R <= 4 ? 2 : 1;                // workers per ring stage
+    static constexpr int kUnitBytes = R * 128 * kRingSubs;       // one worker's words of a tile
+    static constexpr int kStageBytes = kGroup * kUnitBytes;
+    // full mbarriers at 0, empty ones at 128, abort flag at 256, stages filled at 260, zero at 264
     static constexpr int kBarBytes = 512;
     static constexpr int kATabBytes = kDecAreg * 32 * 8;         // per warp: (a_A, a_B) pairs
     static constexpr int kRawBytes = kDecAreg * 32 * 8;          // per warp: raw scales, rows A and B
     static constexpr int kWarpBytes = kATabBytes + kRawBytes;
     // the ring takes what one CTA per SM can have
-    static constexpr int kStagesRaw = (232448 - 1024 - kBarBytes - kRingWarps * kWarpBytes) / kUnitBytes;
+    static constexpr int kStagesRaw = (232448 - 1024 - kBarBytes - kRingWarps * kWarpBytes) / kStageBytes;
     static constexpr int kStages = kStagesRaw > 12 ? 12 : kStagesRaw;
     static constexpr int kRingOff = kBarBytes;
-    static constexpr int kWarpOff = kRingOff + kStages * kUnitBytes;
+    static constexpr int kWarpOff = kRingOff + kStages * kStageBytes;
     static constexpr int kSmem = kWarpOff + kRingWarps * kWarpBytes;
     static_assert(kStages >= 3 && 8 * kStages <= 128, "ring depth fits the barrier area");
 };
@@ -105,13 +110,6 @@ __device__ __forceinline__ void emit8(const DecodeOut& o, uint64_t i, const floa
     }
     if (o.out) stg256(o.out + i, v);
 }
-__device__ __forceinline__ void add_f32_f16x2(uint32_t m, float c, float& lo, float& hi) {
-    asm("{\n\t.reg .b16 h0, h1;\n\t"
-        "mov.b32 {h0, h1}, %2;\n\t"
-        "add.rn.f32.f16 %0, h0, %3;\n\t"
-        "add.rn.f32.f16 %1, h1, %3;\n\t}"
-        : "=f"(lo), "=f"(hi) : "r"(m), "f"(c));
-}
 __device__ __forceinline__ void lds32(uint32_t a, uint32_t& x) {
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x) : "r"(a) : "memory");
 }
@@ -122,17 +120,86 @@ __device__ __forceinline__ void lds128(uint32_t a, uint32_t& x, uint32_t& y, uin
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(a) : "memory");
 }
 
+// Both halves of `m` read as fp16, each plus the fp32 `c`, as fp32: one instruction per half,
+// one rounding (none here: the sums are small integers times a power of two).
+__device__ __forceinline__ void add_f32_f16x2(uint32_t m, float c, float& lo, float& hi) {
+    asm("{\n\t.reg .b16 h0, h1;\n\t"
+        "mov.b32 {h0, h1}, %2;\n\t"
+        "add.rn.f32.f16 %0, h0, %3;\n\t"
+        "add.rn.f32.f16 %1, h1, %3;\n\t}"
+        : "=f"(lo), "=f"(hi) : "r"(m), "f"(c));
+}
+
+// The 64 terms of one worker for the two rows of a lane:
+// acc2[j] <- fma((c_j - s) 2^p_j, (a_A, a_B), acc2[j]), rows A and B in the two halves.
+// subh[i] = -(1024 + s 2^(iR)) (fp16 pair merge); T2[i] = (t, t), t = 2^23 + s 2^(iR)
+// (fp32 merge).  exp_bits: 0x64006400 or 0x4B000000, in a register because a logic
+// instruction takes one immediate, and the field mask is it.
+template <int R>
+__device__ __forceinline__ void ring_pair_terms(const uint32_t (&cwa)[R], const uint32_t (&cwb)[R],
+                                                const uint64_t a2, uint64_t (&acc2)[32],
+                                                const uint32_t exp_bits, const float* subh,
+                                                const uint64_t* T2) {
+    using L = DecodeRing<R>;
+    constexpr uint32_t mask = (1u << R) - 1u;
+    if constexpr (L::kHalf) {
+        constexpr int CW = 32 / R, NF = L::kHalfFields, FV = L::kViewFields;
+#pragma unroll
+        for (int wi = 0; wi < R; ++wi) {
+#pragma unroll
+            for (int v0 = 0; v0 < NF; v0 += FV) {
+                // fields v0 .. v0 + FV - 1 of both halves, brought below bit 10 of each half
+                const uint32_t xa = v0 == 0 ? cwa[wi] : (cwa[wi] >> (v0 * R));
+                const uint32_t xb = v0 == 0 ? cwb[wi] : (cwb[wi] >> (v0 * R));
+#pragma unroll
+                for (int i = 0; i < FV && v0 + i < NF; ++i) {
+                    const uint32_t ma = (xa & ((mask << (i * R)) * 0x00010001u)) | exp_bits;
+                    const uint32_t mb = (xb & ((mask << (i * R)) * 0x00010001u)) | exp_bits;
+                    float la, ha, lb, hb;
+                    add_f32_f16x2(ma, subh[i], la, ha);
+                    add_f32_f16x2(mb, subh[i], lb, hb);
+                    const int jl = wi * CW + v0 + i, jh = jl + NF;
+                    acc2[jl] = fma2(pack2(la, lb), a2, acc2[jl]);
+                    acc2[jh] = fma2(pack2(ha, hb), a2, acc2[jh]);
+                }
+            }
+        }
+    } else {
+        constexpr int FIT = L::kFit;
+        const uint64_t magic2 = ((uint64_t)exp_bits << 32) | exp_bits;
+        // groups of FIT consecutive codes: one funnel shift brings a group's first field to
+        // bit 0, then every field lies below bit 23
+#pragma unroll
+        for (int j0 = 0; j0 < 32; j0 += FIT) {
+            const int bit = j0 * R, wi = bit >> 5, sh = bit & 31;
+            const uint32_t wa = (sh == 0) ? cwa[wi]
+                              : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cwa[wi] >> sh)
+                              : __funnelshift_r(cwa[wi], cwa[wi + 1 < R ? wi + 1 : wi], sh);
+            const uint32_t wb = (sh == 0) ? cwb[wi]
+                              : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cwb[wi] >> sh)
+                              : __funnelshift_r(cwb[wi], cwb[wi + 1 < R ? wi + 1 : wi], sh);
+            const uint64_t w2 = ((uint64_t)wb << 32) | wa;
+#pragma unroll
+            for (int i = 0; i < FIT && j0 + i < 32; ++i) {
+                const uint64_t m2 = ((uint64_t)(mask << (i * R)) << 32) | (uint64_t)(mask << (i * R));
+                // (c - s) 2^(iR) a, rows A and B in one instruction
+                acc2[j0 + i] = fma2(sub2((w2 & m2) | magic2, T2[i]), a2, acc2[j0 + i]);
+            }
+        }
+    }
+}
+
 // What one consumer warp does: its two rows of every tile of the CTA.
 template <int R, bool CARRY>
 __device__ __forceinline__ void decode_ring_consumer(
         const CodecParams& P, const uint32_t W, const MessageTable& tab, const DecodeOut& dst,
-        const uint32_t n_subs, const float w_recip, const int w_pow2, const uint32_t exp23_bits,
+        const uint32_t n_subs, const float w_recip, const int w_pow2, const uint32_t exp_bits,
         const bool first, const bool last, const float w_total, const uint32_t my_tiles,
         const uint32_t wait_limit, const int warp, const int lane, uint8_t* dsm, uint32_t* status) {
     using L = DecodeRing<R>;
     constexpr int S = L::kStages;
     constexpr int FIT = L::kFit;
-    constexpr uint32_t mask = (1u << R) - 1u;
+    constexpr int G = L::kGroup;
     const uint32_t sm0 = smem_u32(dsm);
     const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
     volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 256);
@@ -148,17 +215,13 @@ __device__ __forceinline__ void decode_ring_consumer(
     const uint32_t grp = (lane & ~(gsz - 1)) * kDecAreg;            // my group's first entry
     const uint32_t raw_u32 = smem_u32(raw);
 
-    // 2^23 + s 2^(iR) in both halves: subtracting it from (field | 2^23 bits) leaves
-    // (c - s) 2^(iR)
+    // what turns a merged field into (c - s) 2^p, per field position (see ring_pair_terms)
     uint64_t T2[FIT];
 #pragma unroll
     for (int i = 0; i < FIT; ++i) {
         const float t = __fmaf_rn(P.sf, (float)(1u << (i * R)), 8388608.f);
         T2[i] = pack2(t, t);
     }
-    // the exponent bits arrive as a kernel argument so that they live in a register: a
-    // logic instruction takes one immediate, and the field mask is it
-    const uint64_t magic2 = ((uint64_t)exp23_bits << 32) | exp23_bits;
     float subh[L::kViewFields > 0 ? L::kViewFields : 1];
 #pragma unroll
     for (int i = 0; i < L::kViewFields; ++i) subh[i] = -__fmaf_rn(P.sf, (float)(1u << (i * R)), 1024.f);
@@ -182,51 +245,52 @@ __device__ __forceinline__ void decode_ring_consumer(
     };
     if (my_tiles) fetch_scales(blockIdx.x);
 
-    // ring position of the next unit: stage offset, its barriers' offset, phase
-    uint32_t c_off = 0, c_bar = 0, c_par = 0, held_bar = 0;
+    // ring position of the next stage: byte offset, its barriers' offset, phase
+    uint32_t c_off = 0, c_bar = 0, c_par = 0;
     const uint32_t my_off = sm0 + L::kRingOff + warp * (R * 128) + lane * (R * 4);
-    uint32_t cw[2][R];
-    // Waits for the next unit and copies my two rows' words to registers.  The stage is handed
-    // back only after the words have been used (release_unit): the loads have then certainly
-    // completed, which an arrive issued right behind them does not wait for.  Loading at the
-    // top of every turn keeps the words out of the loop-carried state (carrying them from the
-    // end of the previous turn cost 20 register moves a unit).
-    auto take_unit = [&]() -> bool {
+    uint32_t cw[G][2][R];
+    uint32_t dep = 0;
+    // Waits for the next stage and copies the words of my two rows, for all its workers, to
+    // registers: all loads first, so their latency is met once per stage.  (Loading at the top
+    // of a stage keeps the words out of the loop-carried state: carrying them over from the
+    // previous turn, or fetching a stage ahead into a second register set, costs more in
+    // register moves and control flow than the latency it hides.)
+    auto take_stage = [&]() -> bool {
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_n(bar_full + c_bar, c_par, wait_limit))) return false;
+        constexpr int kStep = (R % 4 == 0) ? 4 : (R % 2 == 0) ? 2 : 1;    // words per load
 #pragma unroll
-        for (int row = 0; row < 2; ++row) {
-            const uint32_t src = my_off + c_off + row * (kRingWarps * R * 128);
-            if constexpr (R % 4 == 0) {
+        for (int k = 0; k < G; ++k) {
 #pragma unroll
-                for (int q = 0; q < R / 4; ++q)
-                    lds128(src + 16 * q, cw[row][4 * q], cw[row][4 * q + 1], cw[row][4 * q + 2], cw[row][4 * q + 3]);
-            } else if constexpr (R % 2 == 0) {
+            for (int row = 0; row < 2; ++row) {
+                const uint32_t src = my_off + c_off + k * L::kUnitBytes + row * (kRingWarps * R * 128);
+                if constexpr (R % 4 == 0) {
 #pragma unroll
-                for (int q = 0; q < R / 2; ++q) lds64(src + 8 * q, cw[row][2 * q], cw[row][2 * q + 1]);
-            } else {
+                    for (int q = 0; q < R / 4; ++q)
+                        lds128(src + 16 * q, cw[k][row][4 * q], cw[k][row][4 * q + 1], cw[k][row][4 * q + 2], cw[k][row][4 * q + 3]);
+                } else if constexpr (R % 2 == 0) {
 #pragma unroll
-                for (int q = 0; q < R; ++q) lds32(src + 4 * q, cw[row][q]);
+                    for (int q = 0; q < R / 2; ++q) lds64(src + 8 * q, cw[k][row][2 * q], cw[k][row][2 * q + 1]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < R; ++q) lds32(src + 4 * q, cw[k][row][q]);
+                }
+#pragma unroll
+                for (int q = 0; q < R; q += kStep) dep ^= cw[k][row][q];
             }
         }
-        held_bar = c_bar;
-        c_off += L::kUnitBytes;
-        c_bar += 8;
-        if (c_bar == 8u * S) { c_off = 0; c_bar = 0; c_par ^= 1u; }
         return true;
     };
-    // `zero` is 0, but only at run time: (x & zero) makes the vote below depend on one word of
-    // every shared load of the unit in every lane, so the loads have completed when it is taken
-    // (a barrier among the lanes alone does not wait for loads in flight).
+    // The stage is handed back only after its words have been used: the loads have then
+    // certainly completed, which an arrive issued right behind them does not wait for.  `zero`
+    // is 0, but only at run time: (dep & zero) makes the arrive depend on one word of every
+    // shared load of the stage (a shared load is one instruction for the whole warp, so lane
+    // 0's dependence covers every lane).
     const uint32_t zero = *reinterpret_cast<volatile uint32_t*>(dsm + 264);
-    auto release_unit = [&]() {
-        constexpr int kStep = (R % 4 == 0) ? 4 : (R % 2 == 0) ? 2 : 1;    // words per load
-        uint32_t x = 0;
-#pragma unroll
-        for (int row = 0; row < 2; ++row)
-#pragma unroll
-            for (int q = 0; q < R; q += kStep) x ^= cw[row][q];
-        const bool done = __all_sync(0xFFFFFFFFu, (x & zero) == 0u);         // always true
-        if (done && lane == 0) mbar_arrive(bar_empty + held_bar);
+    auto release_stage = [&]() {
+        if (lane == 0 && (dep & zero) == 0u) mbar_arrive(bar_empty + c_bar);
+        c_off += L::kStageBytes;
+        c_bar += 8;
+        if (c_bar == 8u * S) { c_off = 0; c_bar = 0; c_par ^= 1u; }
     };
 
     bool ok = true;
@@ -275,55 +339,17 @@ __device__ __forceinline__ void decode_ring_consumer(
             }
         }
 
-        // (four workers per loop turn: 7 % fewer instructions than one per turn; the words are
-        // still loaded at the top of each worker's part)
-#pragma unroll 4
-        for (uint32_t w = 0; w < W; ++w) {
-            if (!take_unit()) { ok = false; break; }
-            const uint64_t a2 = *reinterpret_cast<const uint64_t*>(a_mine + w);       // (a_A, a_B)
-            if constexpr (L::kHalf) {
-                constexpr int CW = 32 / R, NF = L::kHalfFields, FV = L::kViewFields;
+        // the workers in ascending order, a stage (G of them) per turn
+#pragma unroll 2
+        for (uint32_t w0 = 0; w0 < W; w0 += G) {
+            if (!take_stage()) { ok = false; break; }
 #pragma unroll
-                for (int wi = 0; wi < R; ++wi) {
-#pragma unroll
-                    for (int v0 = 0; v0 < NF; v0 += FV) {
-                        const uint32_t xa = v0 == 0 ? cw[0][wi] : (cw[0][wi] >> (v0 * R));
-                        const uint32_t xb = v0 == 0 ? cw[1][wi] : (cw[1][wi] >> (v0 * R));
-#pragma unroll
-                        for (int i = 0; i < FV && v0 + i < NF; ++i) {
-                            const uint32_t ma = (xa & ((mask << (i * R)) * 0x00010001u)) | exp23_bits;
-                            const uint32_t mb = (xb & ((mask << (i * R)) * 0x00010001u)) | exp23_bits;
-                            float la, ha, lb, hb;
-                            add_f32_f16x2(ma, subh[i], la, ha);
-                            add_f32_f16x2(mb, subh[i], lb, hb);
-                            const int jl = wi * CW + v0 + i, jh = jl + NF;
-                            acc2[jl] = fma2(pack2(la, lb), a2, acc2[jl]);
-                            acc2[jh] = fma2(pack2(ha, hb), a2, acc2[jh]);
-                        }
-                    }
-                }
-            } else {
-            // groups of FIT consecutive codes: one funnel shift brings a group's first field
-            // to bit 0, then every field lies below bit 23
-#pragma unroll
-            for (int j0 = 0; j0 < 32; j0 += FIT) {
-                const int bit = j0 * R, wi = bit >> 5, sh = bit & 31;
-                uint32_t word[2];
-#pragma unroll
-                for (int row = 0; row < 2; ++row)
-                    word[row] = (sh == 0) ? cw[row][wi]
-                              : (sh + FIT * R <= 32 || wi + 1 >= R) ? (cw[row][wi] >> sh)
-                              : __funnelshift_r(cw[row][wi], cw[row][wi + 1 < R ? wi + 1 : wi], sh);
-                const uint64_t w2 = ((uint64_t)word[1] << 32) | word[0];
-#pragma unroll
-                for (int i = 0; i < FIT && j0 + i < 32; ++i) {
-                    const uint64_t m2 = ((uint64_t)(mask << (i * R)) << 32) | (uint64_t)(mask << (i * R));
-                    // (c - s) 2^(iR) a, rows A and B in one instruction
-                    acc2[j0 + i] = fma2(sub2((w2 & m2) | magic2, T2[i]), a2, acc2[j0 + i]);
-                }
+            for (int k = 0; k < G; ++k) {
+                if (k > 0 && w0 + k >= W) break;                     // a last, partly filled stage
+                const uint64_t a2 = *reinterpret_cast<const uint64_t*>(a_mine + w0 + k);   // (a_A, a_B)
+                ring_pair_terms<R>(cw[k][0], cw[k][1], a2, acc2, exp_bits, subh, T2);
             }
-            }
-            release_unit();
+            release_stage();
         }
         if (!ok) break;
 
@@ -357,7 +383,7 @@ template <int R, bool CARRY>
 __global__ void __launch_bounds__(kRingThreads, 1)
 decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
                    const DecodeOut dst, const uint32_t n_subs, const uint64_t n_words,
-                   const float w_recip, const int w_pow2, const uint32_t exp23_bits,
+                   const float w_recip, const int w_pow2, const uint32_t exp_bits,
                    const uint32_t wait_limit, const DecodeSlice sl, uint32_t* status) {
     using L = DecodeRing<R>;
     const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
@@ -368,7 +394,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
     const uint32_t sm0 = smem_u32(dsm);
     const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
     volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 256);
-    volatile uint32_t* const s_issued = reinterpret_cast<volatile uint32_t*>(dsm + 260);   // units the producer issued
+    volatile uint32_t* const s_issued = reinterpret_cast<volatile uint32_t*>(dsm + 260);   // stages the producer filled
     const int lane = threadIdx.x & 31;
     // broadcast from lane 0 so that the compiler knows the value is warp-uniform
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
@@ -376,7 +402,6 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
     const uint32_t n_tiles = (n_subs + kRingSubs - 1) / kRingSubs;
     const uint32_t my_tiles =
         blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-    const uint32_t n_units = my_tiles * W;                          // < 2^32: checked by the host
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < S; ++i) {
@@ -391,21 +416,27 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
     __syncthreads();
 
     if (warp == kRingWarps) {
-        // ---- producer: unit n = (my tile n / W, worker n % W), in order, into stage n % S ----
+        // ---- producer: fill n = my n / n_groups-th tile, workers G (n % n_groups) and up, in
+        // order, into stage n % S ----
         if (lane == 0) {
             bool ok = true;
             uint32_t tile = blockIdx.x, w = 0, slot = 0, par = 0, u = 0;
-            for (; u < n_units; ++u) {
+            constexpr int G = L::kGroup;
+            const uint32_t n_fills = my_tiles * ((W + G - 1) / G);
+            for (; u < n_fills; ++u) {
                 // stages are free the first time round; later the consumers hand them back
                 if (u >= (uint32_t)S && !mbar_wait_n(bar_empty + 8 * slot, par ^ 1u, wait_limit)) { ok = false; break; }
                 if (*s_abort) break;                        // a consumer's wait ran out
                 const uint32_t subs = min((uint32_t)kRingSubs, n_subs - tile * kRingSubs);
                 const uint32_t bytes = subs * (R * 128);
+                const uint32_t n = min((uint32_t)G, W - w);
                 const uint32_t bar = bar_full + 8 * slot;
-                mbar_arrive_expect_tx(bar, bytes);
-                bulk_load_1d(sm0 + L::kRingOff + slot * L::kUnitBytes,
-                             tab.codes[w] + (uint64_t)tile * (R * 32 * kRingSubs), bytes, bar);
-                if (++w == W) { w = 0; tile += gridDim.x; }
+                mbar_arrive_expect_tx(bar, n * bytes);
+                for (uint32_t k = 0; k < n; ++k)
+                    bulk_load_1d(sm0 + L::kRingOff + slot * L::kStageBytes + k * L::kUnitBytes,
+                                 tab.codes[w + k] + (uint64_t)tile * (R * 32 * kRingSubs), bytes, bar);
+                w += n;
+                if (w == W) { w = 0; tile += gridDim.x; }
                 if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; }
             }
             *s_issued = u;
@@ -413,13 +444,13 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         }
         __syncwarp();
     } else {
-        decode_ring_consumer<R, CARRY>(P, W, tab, dst, n_subs, w_recip, w_pow2, exp23_bits, first, last,
+        decode_ring_consumer<R, CARRY>(P, W, tab, dst, n_subs, w_recip, w_pow2, exp_bits, first, last,
                                        w_total, my_tiles, wait_limit, warp, lane, dsm, status);
     }
     __syncthreads();
     if (*s_abort) {
         // a wait ran out: let the copies in flight land before the CTA gives its shared memory
-        // back (unit v went into stage v % S; the last S units may still be on their way).
+        // back (fill v went into stage v % S; the last S fills may still be on their way).
         // This wait keeps the full limit whatever the context's.
         if (threadIdx.x == 0) {
             const uint32_t u = *s_issued;
