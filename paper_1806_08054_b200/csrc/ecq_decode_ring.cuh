@@ -135,11 +135,11 @@ __device__ __forceinline__ void add_f32_f16x2(uint32_t m, float c, float& lo, fl
 // subh[i] = -(1024 + s 2^(iR)) (fp16 pair merge); T2[i] = (t, t), t = 2^23 + s 2^(iR)
 // (fp32 merge).  exp_bits: 0x64006400 or 0x4B000000, in a register because a logic
 // instruction takes one immediate, and the field mask is it.
-template <int R>
+template <int R, int NH, int NT>
 __device__ __forceinline__ void ring_pair_terms(const uint32_t (&cwa)[R], const uint32_t (&cwb)[R],
                                                 const uint64_t a2, uint64_t (&acc2)[32],
-                                                const uint32_t exp_bits, const float* subh,
-                                                const uint64_t* T2) {
+                                                const uint32_t exp_bits, const float (&subh)[NH],
+                                                const uint64_t (&T2)[NT]) {
     using L = DecodeRing<R>;
     constexpr uint32_t mask = (1u << R) - 1u;
     if constexpr (L::kHalf) {
@@ -163,6 +163,10 @@ __device__ __forceinline__ void ring_pair_terms(const uint32_t (&cwa)[R], const 
                     acc2[jh] = fma2(pack2(ha, hb), a2, acc2[jh]);
                 }
             }
+            // the sums of this word are due here: keeps the compiler from widening every code
+            // of a worker first and holding 64 of them in registers (no instruction is emitted)
+#pragma unroll
+            for (int j = wi * CW; j < wi * CW + CW; ++j) asm volatile("" : "+l"(acc2[j]));
         }
     } else {
         constexpr int FIT = L::kFit;
@@ -185,6 +189,8 @@ __device__ __forceinline__ void ring_pair_terms(const uint32_t (&cwa)[R], const 
                 // (c - s) 2^(iR) a, rows A and B in one instruction
                 acc2[j0 + i] = fma2(sub2((w2 & m2) | magic2, T2[i]), a2, acc2[j0 + i]);
             }
+#pragma unroll
+            for (int i = 0; i < FIT && j0 + i < 32; ++i) asm volatile("" : "+l"(acc2[j0 + i]));
         }
     }
 }
