@@ -42,6 +42,18 @@ def test_own_arm_line():
     assert set(j["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     m = j["message"]
     assert m["entropy_bound_bits_per_entry"] <= m["fixed_bits_per_entry"] + 1e-9
+    # the receiver kernel: timed inside the step and by itself, against both of its roofs
+    dec = j["decode"]
+    assert dec["ms_per_launch"] > 0 and dec["alone"]["ms_per_launch"] > 0
+    dr = j["decode_roofline"]
+    assert dr["bound"] == "hbm" and abs(dr["frac"] - dr["achieved"] / dr["peak"]) < 1e-9
+    if dr["issue"] is not None:
+        assert dr["issue"]["bound"] == "alu" and 0 < dr["issue"]["frac"] < 1.5
+        assert dr["issue"]["issue_slots_per_code"] == pytest.approx(1 + 1 / 7 + 2)    # r = 3
+    if (os.cpu_count() or 1) > 1:
+        ca = j["cpu_baseline_all_cores"]
+        assert ca["kind"] == "oracle" and ca["cores"] == min(8, os.cpu_count()) and ca["value"] > 0
+    assert "sweep" not in j                                 # only the default workload carries it
 
 
 def test_reference_arm_line():
