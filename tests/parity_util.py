@@ -154,6 +154,37 @@ def sample_ranges(d: int, bucket: int, span: int = 1 << 16, count: int = 3,
     return out
 
 
+def placed_ranges(d: int, bucket: int, W: int, span: int = 8192, count: int = 64,
+                  seed: int = 0) -> List[Tuple[int, int]]:
+    """Whole-bucket windows of about ``span`` entries, placed where the kernels change what
+    they do rather than at random only: the first and last tiles of a vector (in the batched
+    encode launch those are where a CTA passes from one worker's vector to the next), the
+    tiles either side of the points where the grid of CTAs wraps around (encode: 592 and 296
+    CTAs over tiles of 4096 and 8192 entries; receiver: 148 CTAs over tiles of 30720 and 1184
+    warps over tiles of 1024), the last whole tile and the ragged end behind it; random
+    windows fill up to ``count``."""
+    per = max(span // bucket, 1)                       # buckets per window
+    nb = -(-d // bucket)
+    points = [0, d]                                    # entry positions of interest
+    for tile, ctas in ((4096, 592), (8192, 296), (30720, 148), (1024, 1184)):
+        n_t = d // tile
+        points += [tile, tile * ctas, tile * (ctas + 1), 2 * tile * ctas, n_t * tile, (n_t - 1) * tile]
+        # where worker w's share of the launch's global tile sequence meets the grid's stride
+        for w in range(1, min(W, 4)):
+            first = (-(w * n_t)) % ctas                # first tile of worker w that CTA 0 takes
+            points += [first * tile, (first + 1) * tile]
+    starts = set()
+    for pnt in points:
+        b = min(max(pnt // bucket, 0), nb - 1)
+        for b0 in (b - per, b):                        # the window before and the one from the point
+            starts.add(min(max(b0, 0), max(nb - per, 0)))
+    starts.add(max(nb - per, 0))
+    rng = np.random.default_rng(seed)
+    while len(starts) < min(count, max(nb // per, 1)):
+        starts.add(int(rng.integers(0, max(nb - per, 1))))
+    return [(b0 * bucket, min((b0 + per) * bucket, d)) for b0 in sorted(starts)]
+
+
 class SampledOracle:
     """Follows the oracle on sampled whole-bucket ranges of a large vector."""
 
@@ -188,6 +219,38 @@ class SampledOracle:
                                         [self.msgs[w][k][1] for w in range(self.W)],
                                         n=hi - lo, bucket=self.bucket, s=self.s)
             assert close(gpu.out[1][lo:hi].cpu().numpy(), out_or), "decoded mean differs (range %d)" % k
+
+
+def whole_message_properties(gpu: GpuCodec, w: int, grad: torch.Tensor, beta: float,
+                             scratch: torch.Tensor, sum64: torch.Tensor = None):
+    """Worker w's whole message and accumulator after its FIRST encode (h was zero, so the
+    compensated value is the gradient itself), checked on the device over every entry:
+    the dequantised entries g~ (a one-message decode of the codes) are whole multiples q of the
+    bucket's level step a = scale / s with |q| <= s (Eq. 8: every code is in range), lie within
+    one level step of the input (Eq. 9 rounds to a neighbouring level), and the new
+    accumulator is the rounded g - g~ (Eq. 6 with h = 0).  ``sum64`` collects g~ in fp64 for a
+    later check of the decoded mean."""
+    d, B, s = gpu.d, gpu.bucket, gpu.s
+    ecq.ecq_decode_mean(gpu.ctx, [gpu.codes[w][1]], [gpu.scales[w][1]], scratch)
+    assert gpu.status() == ecq.ECQ_OK
+    gq = scratch
+    a = (gpu.scales[w][1] / float(s)).repeat_interleave(B)[:d]
+    live = a > 0
+    # within one level step: Eq. 9 rounds to a neighbouring level; the fp32 roundings of
+    # s/scale, |v| s/scale and q a move the ratio by a few 2^-24 of s levels at most
+    assert bool(((gq - grad).abs() <= a * (1 + s * 2.0 ** -21)).logical_or(~live).all()), "beyond one level step"
+    assert bool((gq[~live] == 0).all())
+    q = torch.where(live, gq / torch.where(live, a, torch.ones_like(a)), torch.zeros_like(gq))
+    qr = q.round()
+    assert bool(((q - qr).abs() <= 1e-4).all()), "a dequantised entry is no multiple of the level step"
+    assert bool((qr.abs() <= s).all()), "level out of range"
+    assert bool((qr * grad >= 0).logical_or(qr == 0).all()), "level with the wrong sign"
+    # Eq. 6 from a zero accumulator: h' = beta * 0 + (g - g~)
+    e = grad - gq
+    h = gpu.err[w][1]
+    assert bool(((h - e).abs() <= ATOL + RTOL * e.abs()).all()), "accumulator is not g - g~"
+    if sum64 is not None:
+        sum64 += gq.double()
 
 
 def whole_vector_properties(gpu: GpuCodec, w: int, grad: torch.Tensor, err_before: torch.Tensor,

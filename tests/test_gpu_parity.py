@@ -7,8 +7,8 @@ import oracle
 import paper_1806_08054_b200 as ecq
 from paper_1806_08054_b200 import workloads as wl
 
-from parity_util import (GpuCodec, SampledOracle, close, codes_np, full_parity, sample_ranges,
-                         whole_vector_properties)
+from parity_util import (GpuCodec, SampledOracle, close, codes_np, full_parity, placed_ranges,
+                         sample_ranges, whole_message_properties, whole_vector_properties)
 
 pytestmark = pytest.mark.gpu
 SEED = wl.CODEC_SEED
@@ -381,10 +381,14 @@ def test_config1_gauss_1m_every_element():
 
 
 def _sampled_config(w, steps, W=None, ranges=None, grads=None):
-    """Full-size run; the oracle follows sampled whole-bucket ranges, and
-    whole-vector properties are checked on the device."""
+    """Full-size run in the launch configuration bench.py times.  The oracle follows placed
+    and random whole-bucket windows of every worker element by element; on the device, over
+    the WHOLE vector of EVERY worker: scales against the library max-abs, and after the first
+    step the message and the accumulator against what Eq. 6, 8 and 9 fix (levels in range,
+    within one level step, accumulator = g - g~), and the decoded mean against the fp64 mean
+    of the dequantised messages."""
     W = W or w.W
-    ranges = ranges or sample_ranges(w.d, w.bucket, seed=w.index)
+    ranges = ranges or placed_ranges(w.d, w.bucket, W, seed=w.index)
     gpu = GpuCodec(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, W)
     so = SampledOracle(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, W, ranges)
     try:
@@ -392,13 +396,31 @@ def _sampled_config(w, steps, W=None, ranges=None, grads=None):
             gs = [grads(p, t) if grads else wl.gradient(w, p, t, "cuda") for p in range(W)]
             before = gpu.err[0][1].clone()
             gpu.encode_batch(t, gs)                 # the launch configuration bench.py times
-            whole_vector_properties(gpu, 0, gs[0], before, w.alpha)
+            if t == 0:
+                zero = torch.zeros_like(before)
+                for p in range(W):
+                    whole_vector_properties(gpu, p, gs[p], zero, w.alpha)
+                del zero
+            else:
+                whole_vector_properties(gpu, 0, gs[0], before, w.alpha)
             del before
+            sum64 = None
+            if t == 0:
+                scratch = torch.empty(w.d, device="cuda")
+                sum64 = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+                for p in range(W):
+                    whole_message_properties(gpu, p, gs[p], w.beta, scratch, sum64)
+                del scratch
             for p in range(W):
                 so.encode_and_compare(gpu, p, t, gs[p])
             del gs
             gpu.decode(W)
             assert gpu.status() == ecq.ECQ_OK
+            if sum64 is not None:
+                mean = sum64 / W
+                assert bool(((gpu.out[1].double() - mean).abs() <= 1e-7 + 1e-6 * mean.abs()).all()), \
+                    "decoded mean is not the mean of the dequantised messages"
+                del sum64, mean
             so.decode_and_compare(gpu)
             gpu.check_guards()
     finally:
@@ -420,6 +442,16 @@ def test_config3_resnet50():
 def test_config4_alexnet():
     w = wl.WORKLOADS["alexnet"]
     _sampled_config(w, steps=w.steps)
+
+
+@pytest.mark.parametrize("name", ["resnet50", "alexnet"])
+def test_config3_and_4_every_element_of_every_worker(name):
+    # one step of the whole configuration against the oracle, element by element, in the
+    # launch configuration bench.py times (batched encode, automatic receiver kernel)
+    w = wl.WORKLOADS[name]
+    full_parity(w.d, w.bucket, w.s, w.alpha, w.beta, SEED, w.W, 1,
+                lambda p, t: wl.gradient(w, p, t, "cuda"), batch=True)
+    torch.cuda.empty_cache()
 
 
 @pytest.mark.parametrize("bucket", wl.LM_SWEEP_BUCKETS)
