@@ -44,7 +44,11 @@ NOMINAL_HBM_GBS = 8000.0
 # levels); commands and counters in profiles/encode_tiled_kernel.md.  Traffic grows in
 # proportion to the entries of a launch, so a full launch's traffic is this figure times its
 # entries.  An entry is dropped (traffic: null) when the kernel changes until it is re-taken.
-NCU_DRAM_BYTES_PER_ENTRY = {}
+NCU_DRAM_BYTES_PER_ENTRY = {      # (bucket, levels): bytes per entry, read + write
+    (512, 4): 10185023744 / 817825024, (128, 1): 9999779584 / 817825024,
+    (4096, 8): 10280564480 / 817825024, (4096, 128): 10688161792 / 817825024,
+    (512, 8): 10285686784 / 817825024, (2048, 1): 9976081408 / 817825024,
+}
 
 
 def code_bits(s: int) -> int:
@@ -565,7 +569,7 @@ def main():
             sr = ecq.ecq_code_bits(sctx)
             senc, sdec = kernel_report(sw, sm, args.sweep_steps, peak, sr)
             eb, db = step_bytes(sw)
-            key = (sw.name, sw.bucket, sw.s)
+            key = (sw.bucket, sw.s)
             sweep.append({"workload": sw.name, "W": sw.W, "d": sw.d, "bucket": sw.bucket, "s": sw.s,
                           "code_bits": sr, "steps": args.sweep_steps,
                           "step_GB/s": (sw.W * eb + db) * args.sweep_steps / (sm["total_ms"] * 1e-3) / 1e9,
@@ -582,7 +586,7 @@ def main():
         step_b = W * enc_bytes + dec_bytes
         value = world * step_b * args.steps / (m["total_ms"] * 1e-3) / 1e9
         enc_obj, dec_obj = kernel_report(w, m, args.steps, peak, r)
-        key = (w.name, w.bucket, w.s)
+        key = (w.bucket, w.s)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": warmup, "ms_per_step": m["total_ms"] / args.steps,

@@ -140,9 +140,8 @@ uint64_t ecq_num_buckets(const ecq_ctx* ctx);
 uint64_t ecq_codes_words(const ecq_ctx* ctx);
 
 /*
- * Sender side, one worker, one iteration (Algorithm 1, "compute quantized local
- * gradients with Eq. 7" and "update the accumulated quantization error with
- * Eq. 6", fused):
+ * Sender side, one worker, one iteration (Algorithm 1, phase 1: the quantisation step,
+ * which applies Eq. 7, and the accumulator step, which applies Eq. 6, fused):
  *   v = grad + alpha*err                            (Eq. 7)
  *   scale_b = max over the bucket of |v_i|          (Eq. 8, l-infinity norm)
  *   level m_i in {floor(x), floor(x)+1}, x = s|v_i|/scale_b, going up with
@@ -167,7 +166,7 @@ int ecq_encode(ecq_ctx* ctx, uint32_t worker, uint32_t step, const float* grad,
 
 /*
  * ecq_encode for workers 0..W-1 of one iteration in ONE kernel launch (Algorithm 1,
- * the loop "for p = 1..P" of phase 1, on a single GPU that holds all P workers'
+ * the loop over the P nodes of phase 1, on a single GPU that holds all P workers'
  * slices).  Results are identical to W calls of ecq_encode(ctx, w, step, grads[w],
  * errs[w], codes[w], scales[w]); a single launch spares W-1 launch ramps and tails,
  * which matters for vectors of tens of megabytes.  Beyond ECQ_MAX_WORKERS workers there
@@ -182,7 +181,7 @@ int ecq_encode_batch(ecq_ctx* ctx, uint32_t W, uint32_t step, const float* const
                      void* cuda_stream);
 
 /*
- * Receiver side (Eq. 4 and Algorithm 1, "compute global gradients"):
+ * Receiver side (Eq. 4 and Algorithm 1, phase 2, global-gradient step):
  *   out_i = (1/W) * sum_{w<W} q_{w,i} * (scales_w[b(i)] / s)
  *   W       number of messages, 1..ECQ_MAX_WORKERS_TOTAL
  *   codes   HOST array of W device pointers to the workers' code streams
@@ -198,8 +197,8 @@ int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
                     const float* const* scales, float* out, void* cuda_stream);
 
 /*
- * Receiver side with the model update fused in (Algorithm 1, "compute global
- * gradients" followed by "update model parameters w(t+1) = w(t) - eta * g~(t)"):
+ * Receiver side with the model update fused in (Algorithm 1, phase 2: the global-gradient
+ * step followed by the model-update step, w(t+1) = w(t) - eta * g~(t)):
  *   g~_i     = the mean ecq_decode_mean would produce
  *   params_i <- fma(-eta, g~_i, params_i)       (one rounding)
  *   out_i    = g~_i when out is not NULL
@@ -226,7 +225,7 @@ double ecq_entropy_bound_bits(const uint64_t* counts_host, uint32_t n_bins);
 
 /*
  * Entropy-coded message.  The paragraph after Eq. 9 notes that the r-bit codes can be
- * compressed further by an entropy code ("e.g. Huffman") with at most
+ * compressed further by an entropy code (the paper names Huffman coding as one) with at most
  * sum_k d_k log2(d / d_k) bits, and the linear-model experiments count their
  * communication that way.  The paper fixes no format; this one is the library's:
  *   - a prefix code over the 2s+1 level indices, optimal among codes whose words have at

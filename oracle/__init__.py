@@ -7,7 +7,7 @@ and its Python binding never do, and this package imports nothing of theirs.
 
 Functions follow the paper's Section 4: ``encode`` is Eq. 7 + Eq. 8 (l-infinity
 scale per bucket) + Eq. 9 + Eq. 6 + the fixed-width code; ``decode_mean`` is
-Eq. 4 / the "compute global gradients" line of Algorithm 1.
+Eq. 4 / the global-gradient step of Algorithm 1's phase 2.
 """
 from __future__ import annotations
 

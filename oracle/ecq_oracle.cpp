@@ -13,7 +13,7 @@
 //                scale taken per bucket, Eq. 9 (two-point stochastic rounding),
 //                Eq. 6 (incremental error accumulator), and the fixed-width
 //                r = ceil(log2(2s+1)) bit code of the paragraph after Eq. 9.
-//   decode_mean  Eq. 4 / Algorithm 1 "compute global gradients": the mean of
+//   decode_mean  Eq. 4 / Algorithm 1, phase 2, global-gradient step: the mean of
 //                the P dequantised messages.
 //
 // The paper works over the reals.  Every fp32 rounding decision below is a
@@ -23,7 +23,7 @@
 // Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11), written
 // here from its published round function.
 //
-//   decode_mean_update  the same followed by Algorithm 1's "update model parameters".
+//   decode_mean_update  the same followed by Algorithm 1's model-update step.
 //
 // Parity pins (tests/test_oracle_*.py): Philox known answers; closed forms for
 // r and the message length; hand-worked level-boundary inputs; exact-rational
@@ -250,7 +250,7 @@ int ecqo_encode_given_draws(uint64_t n, uint32_t B, uint32_t s, float alpha, flo
                        codes, scales, status);
 }
 
-// Eq. 4 / Algorithm 1 "compute global gradients": out_i = (1/W) sum_w q_{w,i} a_{w,b},
+// Eq. 4 / Algorithm 1, phase 2, global-gradient step: out_i = (1/W) sum_w q_{w,i} a_{w,b},
 // a_{w,b} = scale_{w,b}/s, summed in ascending w, then one division by W.
 int ecqo_decode_mean(uint64_t n, uint32_t B, uint32_t s, uint32_t W,
                      const uint32_t* const* codes, const float* const* scales,
@@ -271,7 +271,7 @@ int ecqo_decode_mean(uint64_t n, uint32_t B, uint32_t s, uint32_t W,
     return 0;
 }
 
-// Algorithm 1, "update model parameters": w <- w - eta * g~, with g~ the mean above,
+// Algorithm 1, phase 2, model-update step: w <- w - eta * g~, with g~ the mean above,
 // as one fused multiply-add per entry.
 int ecqo_decode_mean_update(uint64_t n, uint32_t B, uint32_t s, uint32_t W,
                             const uint32_t* const* codes, const float* const* scales,

@@ -1,5 +1,5 @@
-// Receiver-side kernel: unpack -> dequantise -> W-way mean (Eq. 4; Algorithm 1,
-// "compute global gradients").
+// Receiver-side kernel: unpack -> dequantise -> W-way mean (Eq. 4; Algorithm 1, phase 2,
+// global-gradient step).
 #pragma once
 
 #include "ecq_common.cuh"
@@ -12,7 +12,7 @@ struct MessageTable {
 };
 
 // Where a decoded mean goes: to `out` (may be null), and, for the fused model update of
-// Algorithm 1 ("update model parameters w <- w - eta * g~"), into `params` (may be null).
+// Algorithm 1 (phase 2, model-update step: w <- w - eta * g~), into `params` (may be null).
 // More than 64 messages are summed over several launches of 64: every launch but the first
 // starts from the running sums a previous one left in `out` (first == 0), and every launch
 // but the last leaves its running sums there instead of the mean (last == 0).  The chain of

@@ -1,5 +1,6 @@
-// Entropy-coded message (paragraph after Eq. 9: the r-bit codes "can be further compressed
-// by entropy coding, e.g. Huffman"; the linear-model experiments count bits that way).
+// Entropy-coded message (paragraph after Eq. 9: the r-bit codes may be compressed further by
+// an entropy code, Huffman coding being the one named; the linear-model experiments count
+// bits that way).
 //
 // Format: canonical prefix code over the 2s+1 level indices with words of at most 12 bits;
 // a word's bits enter the stream in tree order, first bit in the lowest free bit of the
