@@ -288,22 +288,24 @@ bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeO
     auto kern = decode_ring_kernel<R, CARRY>;
     std::call_once(once[dev], [&] {
         int o = 0;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kSmem) ==
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kMaxSmem) ==
                 cudaSuccess &&
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kRingThreads, L::kSmem) ==
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, kRingThreads, L::kMaxSmem) ==
                 cudaSuccess)
             occ[dev] = o;
     });
     if (occ[dev] <= 0) return false;
+    const RingLayout lay = ring_layout<R>(W, B);
+    if (lay.stages < 3) return false;
     uint32_t grid = (uint32_t)(c->sm_count * occ[dev]);
     if (c->decode_kernel == ECQ_DECODE_AUTO &&
         (n_tiles < (uint64_t)kRingMinTilesPerCta * grid || R > kRingMaxAutoBits))
         return false;
     if (c->decode_max_ctas && grid > c->decode_max_ctas) grid = c->decode_max_ctas;
     if (grid > n_tiles) grid = (uint32_t)n_tiles;
-    kern<<<grid, kRingThreads, L::kSmem, st>>>(c->P, W, tab, out, (uint32_t)n_subs64, c->n_words,
-                                                  w_recip, w_pow2, L::kHalf ? 0x64006400u : 0x4B000000u,
-                                                  c->wait_limit, sl, c->d_status);
+    kern<<<grid, kRingThreads, lay.smem, st>>>(c->P, W, tab, out, (uint32_t)n_subs64, c->n_words,
+                                               w_recip, w_pow2, L::kHalf ? 0x64006400u : 0x4B000000u,
+                                               c->wait_limit, lay, sl, c->d_status);
     return true;
 }
 

@@ -62,17 +62,34 @@ template <int R> struct DecodeRing {
     static constexpr int kStageBytes = kGroup * kUnitBytes;
     // full mbarriers at 0, empty ones at 128, abort flag at 256, stages filled at 260, zero at 264
     static constexpr int kBarBytes = 512;
-    static constexpr int kATabBytes = kDecAreg * 32 * 8;         // per warp: (a_A, a_B) pairs
-    static constexpr int kRawBytes = kDecAreg * 32 * 8;          // per warp: raw scales, rows A and B
-    static constexpr int kWarpBytes = kATabBytes + kRawBytes;
-    // the ring takes what one CTA per SM can have
-    static constexpr int kStagesRaw = (232448 - 1024 - kBarBytes - kRingWarps * kWarpBytes) / kStageBytes;
-    static constexpr int kStages = kStagesRaw > 12 ? 12 : kStagesRaw;
     static constexpr int kRingOff = kBarBytes;
-    static constexpr int kWarpOff = kRingOff + kStages * kStageBytes;
-    static constexpr int kSmem = kWarpOff + kRingWarps * kWarpBytes;
-    static_assert(kStages >= 3 && 8 * kStages <= 128, "ring depth fits the barrier area");
+    static constexpr int kMaxSmem = 232448 - 1024;               // what one CTA per SM can have
+    static constexpr int kMaxStages = 12;                        // 16 barriers fit each barrier area
 };
+
+// Shared memory of one launch: the ring takes what the level-step tables leave.  A consumer
+// warp keeps, per group of lanes that share a bucket, `wstride` entries of (a_A, a_B) and as
+// many raw scale pairs: 16 bytes per entry, (32 / gsz) groups.  (With every table at its
+// largest, 4 KB a warp, the ring would lose 46 KB; its depth is worth 3-4 % a stage.)
+struct RingLayout {
+    uint32_t wstride;        // table entries per lane group: the workers of the launch, even
+    uint32_t warp_bytes;     // tables of one consumer warp
+    uint32_t stages;         // ring depth
+    uint32_t smem;           // dynamic shared memory of the launch
+};
+template <int R>
+inline RingLayout ring_layout(uint32_t W, uint32_t bucket) {
+    using L = DecodeRing<R>;
+    const uint32_t gsz = bucket >= 1024u ? 32u : (bucket >> 5);
+    RingLayout y;
+    y.wstride = (W + 1u) & ~1u;
+    y.warp_bytes = (32u / gsz) * y.wstride * 16u;
+    const uint32_t room = (uint32_t)L::kMaxSmem - (uint32_t)L::kRingOff - (uint32_t)kRingWarps * y.warp_bytes;
+    y.stages = room / (uint32_t)L::kStageBytes;
+    if (y.stages > (uint32_t)L::kMaxStages) y.stages = (uint32_t)L::kMaxStages;
+    y.smem = (uint32_t)L::kRingOff + y.stages * (uint32_t)L::kStageBytes + (uint32_t)kRingWarps * y.warp_bytes;
+    return y;
+}
 
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
@@ -201,24 +218,27 @@ __device__ __forceinline__ void decode_ring_consumer(
         const CodecParams& P, const uint32_t W, const MessageTable& tab, const DecodeOut& dst,
         const uint32_t n_subs, const float w_recip, const int w_pow2, const uint32_t exp_bits,
         const bool first, const bool last, const float w_total, const uint32_t my_tiles,
-        const uint32_t wait_limit, const int warp, const int lane, uint8_t* dsm, uint32_t* status) {
+        const uint32_t wait_limit, const RingLayout lay, const int warp, const int lane, uint8_t* dsm,
+        uint32_t* status) {
     using L = DecodeRing<R>;
-    constexpr int S = L::kStages;
+    const uint32_t S = lay.stages;
     constexpr int FIT = L::kFit;
     constexpr int G = L::kGroup;
     const uint32_t sm0 = smem_u32(dsm);
     const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
     volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 256);
-    float2* const a_tab = reinterpret_cast<float2*>(dsm + L::kWarpOff + warp * L::kWarpBytes);
-    float* const raw = reinterpret_cast<float*>(dsm + L::kWarpOff + warp * L::kWarpBytes + L::kATabBytes);
+    uint8_t* const my_tabs = dsm + L::kRingOff + S * L::kStageBytes + warp * lay.warp_bytes;
+    float2* const a_tab = reinterpret_cast<float2*>(my_tabs);
+    float* const raw = reinterpret_cast<float*>(my_tabs + lay.warp_bytes / 2);
 
     // lanes that share a bucket: gsz consecutive lanes (all 32 from 1024 entries up); a_tab
-    // holds, per group of lanes, (a_w of row A, a_w of row B) for w < W (W <= kDecAreg * gsz)
+    // holds, per group of lanes, (a_w of row A, a_w of row B) for w < W (W <= kDecAreg * gsz),
+    // lay.wstride entries a group
     const uint32_t gsz = P.bucket >= 1024u ? 32u : (P.bucket >> 5);
     const uint32_t gl = lane & (gsz - 1);
     const uint32_t bucket_shift = 31 - __clz(P.bucket);           // bucket is a power of two
     const uint32_t n_slots = (W + gsz - 1) / gsz;                   // <= kDecAreg
-    const uint32_t grp = (lane & ~(gsz - 1)) * kDecAreg;            // my group's first entry
+    const uint32_t grp = ((uint32_t)lane / gsz) * lay.wstride;       // my group's first entry
     const uint32_t raw_u32 = smem_u32(raw);
 
     // what turns a merged field into (c - s) 2^p, per field position (see ring_pair_terms)
@@ -390,11 +410,11 @@ __global__ void __launch_bounds__(kRingThreads, 1)
 decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant__ MessageTable tab,
                    const DecodeOut dst, const uint32_t n_subs, const uint64_t n_words,
                    const float w_recip, const int w_pow2, const uint32_t exp_bits,
-                   const uint32_t wait_limit, const DecodeSlice sl, uint32_t* status) {
+                   const uint32_t wait_limit, const RingLayout lay, const DecodeSlice sl, uint32_t* status) {
     using L = DecodeRing<R>;
     const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
     const float w_total = CARRY ? sl.w_total : (float)W;
-    constexpr int S = L::kStages;
+    const uint32_t S = lay.stages;
     constexpr uint32_t mask = (1u << R) - 1u;
     extern __shared__ __align__(128) uint8_t dsm[];
     const uint32_t sm0 = smem_u32(dsm);
@@ -410,7 +430,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < S; ++i) {
+        for (uint32_t i = 0; i < S; ++i) {
             mbar_init(bar_full + 8 * i, 1);
             mbar_init(bar_empty + 8 * i, kRingWarps);
         }
@@ -431,7 +451,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
             const uint32_t n_fills = my_tiles * ((W + G - 1) / G);
             for (; u < n_fills; ++u) {
                 // stages are free the first time round; later the consumers hand them back
-                if (u >= (uint32_t)S && !mbar_wait_n(bar_empty + 8 * slot, par ^ 1u, wait_limit)) { ok = false; break; }
+                if (u >= S && !mbar_wait_n(bar_empty + 8 * slot, par ^ 1u, wait_limit)) { ok = false; break; }
                 if (*s_abort) break;                        // a consumer's wait ran out
                 const uint32_t subs = min((uint32_t)kRingSubs, n_subs - tile * kRingSubs);
                 const uint32_t bytes = subs * (R * 128);
@@ -443,7 +463,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
                                  tab.codes[w + k] + (uint64_t)tile * (R * 32 * kRingSubs), bytes, bar);
                 w += n;
                 if (w == W) { w = 0; tile += gridDim.x; }
-                if (++slot == (uint32_t)S) { slot = 0; par ^= 1u; }
+                if (++slot == S) { slot = 0; par ^= 1u; }
             }
             *s_issued = u;
             if (!ok) { *s_abort = 1; atomicOr(status, kStatusTimeout); }    // a stage never came back
@@ -451,7 +471,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         __syncwarp();
     } else {
         decode_ring_consumer<R, CARRY>(P, W, tab, dst, n_subs, w_recip, w_pow2, exp_bits, first, last,
-                                       w_total, my_tiles, wait_limit, warp, lane, dsm, status);
+                                       w_total, my_tiles, wait_limit, lay, warp, lane, dsm, status);
     }
     __syncthreads();
     if (*s_abort) {
@@ -460,7 +480,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         // This wait keeps the full limit whatever the context's.
         if (threadIdx.x == 0) {
             const uint32_t u = *s_issued;
-            for (uint32_t v = (u > (uint32_t)S ? u - S : 0); v < u; ++v)
+            for (uint32_t v = (u > S ? u - S : 0); v < u; ++v)
                 mbar_wait(bar_full + 8 * (v % S), (v / S) & 1u);
         }
         return;
