@@ -65,6 +65,11 @@ template <int R> struct DecodeRing {
     static constexpr int kRingOff = kBarBytes;
     static constexpr int kMaxSmem = 232448 - 1024;               // what one CTA per SM can have
     static constexpr int kMaxStages = 12;                        // 16 barriers fit each barrier area
+    // at two bits the kernel is shortest of registers: ring depth and table strides stay
+    // compile-time constants there (worst-case tables of 4 KB a warp; measured 2 % faster)
+    static constexpr bool kFixedLayout = R == 2;
+    static constexpr int kFixedStages = (kMaxSmem - kRingOff - kRingWarps * kDecAreg * 32 * 16) / kStageBytes > kMaxStages
+        ? kMaxStages : (kMaxSmem - kRingOff - kRingWarps * kDecAreg * 32 * 16) / kStageBytes;
 };
 
 // Shared memory of one launch: the ring takes what the level-step tables leave.  A consumer
@@ -83,6 +88,7 @@ inline RingLayout ring_layout(uint32_t W, uint32_t bucket) {
     const uint32_t gsz = bucket >= 1024u ? 32u : (bucket >> 5);
     RingLayout y;
     y.wstride = (W + 1u) & ~1u;
+    if (L::kFixedLayout) y.wstride = (uint32_t)kDecAreg * gsz;       // 4 KB a warp whatever the launch
     y.warp_bytes = (32u / gsz) * y.wstride * 16u;
     const uint32_t room = (uint32_t)L::kMaxSmem - (uint32_t)L::kRingOff - (uint32_t)kRingWarps * y.warp_bytes;
     y.stages = room / (uint32_t)L::kStageBytes;
@@ -221,15 +227,16 @@ __device__ __forceinline__ void decode_ring_consumer(
         const uint32_t wait_limit, const RingLayout lay, const int warp, const int lane, uint8_t* dsm,
         uint32_t* status) {
     using L = DecodeRing<R>;
-    const uint32_t S = lay.stages;
+    const uint32_t S = L::kFixedLayout ? (uint32_t)L::kFixedStages : lay.stages;
     constexpr int FIT = L::kFit;
     constexpr int G = L::kGroup;
     const uint32_t sm0 = smem_u32(dsm);
     const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
     volatile uint32_t* const s_abort = reinterpret_cast<volatile uint32_t*>(dsm + 256);
-    uint8_t* const my_tabs = dsm + L::kRingOff + S * L::kStageBytes + warp * lay.warp_bytes;
+    const uint32_t warp_bytes = L::kFixedLayout ? (uint32_t)kDecAreg * 32 * 16 : lay.warp_bytes;
+    uint8_t* const my_tabs = dsm + L::kRingOff + S * L::kStageBytes + warp * warp_bytes;
     float2* const a_tab = reinterpret_cast<float2*>(my_tabs);
-    float* const raw = reinterpret_cast<float*>(my_tabs + lay.warp_bytes / 2);
+    float* const raw = reinterpret_cast<float*>(my_tabs + warp_bytes / 2);
 
     // lanes that share a bucket: gsz consecutive lanes (all 32 from 1024 entries up); a_tab
     // holds, per group of lanes, (a_w of row A, a_w of row B) for w < W (W <= kDecAreg * gsz),
@@ -238,7 +245,7 @@ __device__ __forceinline__ void decode_ring_consumer(
     const uint32_t gl = lane & (gsz - 1);
     const uint32_t bucket_shift = 31 - __clz(P.bucket);           // bucket is a power of two
     const uint32_t n_slots = (W + gsz - 1) / gsz;                   // <= kDecAreg
-    const uint32_t grp = ((uint32_t)lane / gsz) * lay.wstride;       // my group's first entry
+    const uint32_t grp = L::kFixedLayout ? (lane & ~(gsz - 1)) * kDecAreg : ((uint32_t)lane / gsz) * lay.wstride;   // my group's first entry
     const uint32_t raw_u32 = smem_u32(raw);
 
     // what turns a merged field into (c - s) 2^p, per field position (see ring_pair_terms)
@@ -414,7 +421,7 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
     using L = DecodeRing<R>;
     const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
     const float w_total = CARRY ? sl.w_total : (float)W;
-    const uint32_t S = lay.stages;
+    const uint32_t S = L::kFixedLayout ? (uint32_t)L::kFixedStages : lay.stages;
     constexpr uint32_t mask = (1u << R) - 1u;
     extern __shared__ __align__(128) uint8_t dsm[];
     const uint32_t sm0 = smem_u32(dsm);
