@@ -323,7 +323,61 @@ def issue_slots_per_code(r: int) -> float:
     return 1.0 + 1.0 / fit + 1.0 + 1.0
 
 
-def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world):
+def decode_length_ladder(ecq, w, codes, scales, out):
+    """The receiver kernels on prefixes of the resident messages, to separate what a launch
+    costs whatever its length from what it costs per output.  A prefix of k rounds is
+    k x (one long-vector tile of 30720 outputs per SM) outputs; its code words and scales are
+    the first words and scales of every worker's message (whole buckets, whole words).  Each
+    kernel is forced by name, timed by itself with L2 flushed before every launch (the short
+    prefixes would fit in it), and the medians are fitted by a line: time = fixed + rounds x
+    per_round.  Returns None when the vector is shorter than two rounds."""
+    import statistics
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    per_round = sms * 30720
+    if per_round % w.bucket or w.d < 2 * per_round:
+        return None
+    r = code_bits(w.s)
+    ks = [k for k in (1, 2, 3, 4, 6, 8, 12, 16) if k * per_round <= w.d]
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
+    res = {"entries_per_round": per_round, "rounds": ks,
+           "timed": "each prefix by itself, median of 9 launches, L2 flushed before each"}
+    _, dec_bytes_round = step_bytes(wl.Workload(w.name, w.index, w.W, per_round, w.bucket, w.s,
+                                                w.alpha, w.beta, 1, w.kind))
+    for name, kernel in (("ring", ecq.ECQ_DECODE_RING), ("warp", ecq.ECQ_DECODE_WARP)):
+        if kernel == ecq.ECQ_DECODE_RING and r > 9:
+            continue
+        us = []
+        for k in ks:
+            n = k * per_round
+            c = ecq.ecq_create(n, w.bucket, w.s, w.alpha, w.beta, wl.CODEC_SEED)
+            ecq.ecq_set_decode_plan(c, kernel, 0)
+            cs = [x[:n * r // 32] for x in codes]
+            ss = [x[:n // w.bucket] for x in scales]
+            o = out[:n]
+            ts = []
+            for i in range(12):
+                flush.fill_(i)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                ecq.ecq_decode_mean(c, cs, ss, o)
+                b.record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b) * 1e3)
+            if ecq.ecq_status(c) != ecq.ECQ_OK:
+                raise SystemExit("codec status on a prefix of %d entries" % n)
+            ecq.ecq_destroy(c)
+            us.append(statistics.median(ts))
+        # least squares line through (rounds, microseconds)
+        mk, mu = sum(ks) / len(ks), sum(us) / len(us)
+        slope = sum((k - mk) * (u - mu) for k, u in zip(ks, us)) / sum((k - mk) ** 2 for k in ks)
+        res[name] = {"us": us, "us_per_round": slope, "fixed_us": mu - slope * mk,
+                     "per_round_GB/s": dec_bytes_round / (slope * 1e-6) / 1e9}
+    del flush
+    return res
+
+
+def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, ladder_wanted=True):
     """Times `steps` steps (batched encode + decode-mean) of workload `w` on resident
     buffers; returns per-kernel times (max over ranks), the launches made and the clocks
     sampled meanwhile."""
@@ -388,9 +442,10 @@ def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world):
     status = ecq.ecq_status(ctx)
     if status != ecq.ECQ_OK:
         raise SystemExit("codec status %d: %s" % (status, ecq.binding.strerror(status)))
+    ladder = decode_length_ladder(ecq, w, codes, scales, out) if (ladder_wanted and world == 1) else None
     total_ms, enc_ms, dec_ms, alone_ms = max_over_ranks([total_ms, enc_ms, dec_ms, alone_ms], world)
     return {"total_ms": total_ms, "enc_ms": enc_ms, "dec_ms": dec_ms, "alone_ms": alone_ms,
-            "launches": int(launches), "clocks": clocks, "clocks_alone": clocks2,
+            "launches": int(launches), "clocks": clocks, "clocks_alone": clocks2, "ladder": ladder,
             "codes": codes, "scales": scales, "out": out}
 
 
@@ -415,7 +470,8 @@ def kernel_report(w, m, steps, peak, r):
                      "frac_of_measured_copy": alone_gbs / peak,
                      "frac_of_nominal_8TBs": alone_gbs / NOMINAL_HBM_GBS,
                      "sm_mhz": mhz2, "ms_x_sm_ghz": m["alone_ms"] * mhz2 / 1e3 if mhz2 else None,
-                     "timed": "launches back to back after the timed steps and 0.3 s of idle"}}
+                     "timed": "launches back to back after the timed steps and 0.3 s of idle"},
+           "length_ladder": m.get("ladder")}
     # The receiver's second roof: instruction issue.  Codes per second that 148 x 4 warp
     # schedulers issue at the SM clock sampled during the launches, at the slots per code of
     # the kernel's arithmetic (issue_slots_per_code); nothing but that arithmetic is counted,
@@ -452,6 +508,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true",
                     help="skip the other >= 25 M-entry configurations (default workload only)")
     ap.add_argument("--no-message", action="store_true", help="skip the entropy-coded message figures")
+    ap.add_argument("--no-ladder", action="store_true",
+                    help="skip the receiver's time-against-length ladder")
     ap.add_argument("--sweep-steps", type=int, default=5)
     ap.add_argument("--cpu-elems", type=int, default=1 << 25)
     ap.add_argument("--ref-elems", type=int, default=1 << 22)
@@ -499,7 +557,8 @@ def main():
     errs = [err[p * d:(p + 1) * d] for p in range(W)]
     grad_list = [grads[p % G] for p in range(W)]
 
-    m = measure(ecq, ctx, w, grad_list, errs, args.steps, warmup, rank, local, world)
+    m = measure(ecq, ctx, w, grad_list, errs, args.steps, warmup, rank, local, world,
+                ladder_wanted=not args.no_ladder)
     codes = m["codes"]
     # level statistics of worker 0's last message (outside the timed region)
     message = None
@@ -564,7 +623,8 @@ def main():
                 sgrads = own
             err.zero_()
             serrs = [err[p * sw.d:(p + 1) * sw.d] for p in range(sw.W)]
-            sm = measure(ecq, sctx, sw, sgrads, serrs, args.sweep_steps, 3, rank, local, world)
+            sm = measure(ecq, sctx, sw, sgrads, serrs, args.sweep_steps, 3, rank, local, world,
+                         ladder_wanted=not args.no_ladder)
             sm.pop("codes"), sm.pop("scales"), sm.pop("out")
             sr = ecq.ecq_code_bits(sctx)
             senc, sdec = kernel_report(sw, sm, args.sweep_steps, peak, sr)

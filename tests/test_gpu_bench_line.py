@@ -54,10 +54,17 @@ def test_own_arm_line():
         ca = j["cpu_baseline_all_cores"]
         assert ca["kind"] == "oracle" and ca["cores"] == min(8, os.cpu_count()) and ca["value"] > 0
     assert "sweep" not in j                                 # only the default workload carries it
+    assert dec["length_ladder"] is None                     # shorter than two rounds of long-vector tiles
 
 
-def test_reference_arm_line():
-    j = _run("--impl", "reference", "--workload", "lsq_4m", "--steps", "1", "--warmup", "0",
-             "--ref-elems", "65536")
-    assert j["impl"] == "reference" and j["metric"] == "codec_step_throughput" and j["value"] > 0
-    assert j["cpu_baseline"]["kind"] == "oracle" and j["e2e"]["h2d_bytes_per_step"] == 0
+def test_receiver_length_ladder_on_a_mid_size_workload():
+    j = _run("--workload", "resnet50", "--steps", "3", "--warmup", "3", "--no-e2e", "--no-cpu",
+             "--no-message")
+    lad = j["decode"]["length_ladder"]
+    assert lad["rounds"] == [1, 2, 3, 4] and lad["entries_per_round"] % 30720 == 0
+    for name in ("ring", "warp"):
+        k = lad[name]
+        assert len(k["us"]) == 4 and all(u > 0 for u in k["us"])
+        assert k["us"][-1] > k["us"][0] and k["us_per_round"] > 0 and k["per_round_GB/s"] > 0
+    j = _run("--workload", "resnet50", "--steps", "3", "--no-e2e", "--no-cpu", "--no-message", "--no-ladder")
+    assert j["decode"]["length_ladder"] is None
