@@ -377,6 +377,35 @@ def decode_length_ladder(ecq, w, codes, scales, out):
     return res
 
 
+def graph_replay(ecq, ctx, w, t_g, t_h, t_c, t_s, out, steps, first_step):
+    """`steps` steps (each with its own step index) captured into one CUDA graph and replayed:
+    what the GPU takes for them when the host's launch calls are out of the way.  For the
+    workloads that fit in L2, where a step is shorter than the host's launch calls."""
+    try:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for t in range(steps):
+                ecq.ecq_encode_batch(ctx, first_step + t, t_g, t_h, t_c, t_s)
+                ecq.ecq_decode_mean(ctx, t_c, t_s, out)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        reps = 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+    except RuntimeError as exc:                          # capture refused: report, do not fail
+        return {"unavailable": str(exc).splitlines()[0][:200]}
+    ms = e0.elapsed_time(e1) / (reps * steps)
+    enc_b, dec_b = step_bytes(w)
+    return {"ms_per_step": ms, "GB/s": (w.W * enc_b + dec_b) / (ms * 1e-3) / 1e9,
+            "steps_per_graph": steps, "replays": reps,
+            "timed": "one CUDA graph of the steps' launches, replayed back to back"}
+
+
 def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, ladder_wanted=True):
     """Times `steps` steps (batched encode + decode-mean) of workload `w` on resident
     buffers; returns per-kernel times (max over ranks), the launches made and the clocks
@@ -387,12 +416,16 @@ def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, lad
     scales = [torch.zeros(nb, device="cuda") for _ in range(W)]
     out = torch.zeros(d, device="cuda")
 
+    # the buffers are the same in every step: their addresses are marshalled once
+    t_g, t_h = ecq.pointer_table(grad_list, torch.float32, "grads"), ecq.pointer_table(errs, torch.float32, "errs")
+    t_c, t_s = ecq.pointer_table(codes, torch.int32, "codes"), ecq.pointer_table(scales, torch.float32, "scales")
+
     def step(t):
         # all W workers' encodes as one batched launch, then the decode-mean
-        ecq.ecq_encode_batch(ctx, t, grad_list, errs, codes, scales)
+        ecq.ecq_encode_batch(ctx, t, t_g, t_h, t_c, t_s)
         ev_mid = torch.cuda.Event(enable_timing=True)
         ev_mid.record()
-        ecq.ecq_decode_mean(ctx, codes, scales, out)
+        ecq.ecq_decode_mean(ctx, t_c, t_s, out)
         return ev_mid
 
     for t in range(warmup):
@@ -426,7 +459,7 @@ def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, lad
     n_alone = max(3, min(20, int(4.0 / max(dec_ms / steps, 1e-3))))
     time.sleep(0.3)
     for _ in range(2):
-        ecq.ecq_decode_mean(ctx, codes, scales, out)
+        ecq.ecq_decode_mean(ctx, t_c, t_s, out)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler2 = ClockSampler(local)
@@ -434,7 +467,7 @@ def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, lad
         sampler2.start()
     e0.record()
     for _ in range(n_alone):
-        ecq.ecq_decode_mean(ctx, codes, scales, out)
+        ecq.ecq_decode_mean(ctx, t_c, t_s, out)
     e1.record()
     torch.cuda.synchronize()
     clocks2 = sampler2.stop() if rank == 0 else None
@@ -443,9 +476,16 @@ def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, lad
     if status != ecq.ECQ_OK:
         raise SystemExit("codec status %d: %s" % (status, ecq.binding.strerror(status)))
     ladder = decode_length_ladder(ecq, w, codes, scales, out) if (ladder_wanted and world == 1) else None
+    enc_b, dec_b = step_bytes(w)
+    graph = (graph_replay(ecq, ctx, w, t_g, t_h, t_c, t_s, out, steps, warmup + steps)
+             if world == 1 and W * enc_b + dec_b <= 4 * 126e6 else None)
+    status = ecq.ecq_status(ctx)
+    if status != ecq.ECQ_OK:
+        raise SystemExit("codec status %d after the graph replays" % status)
     total_ms, enc_ms, dec_ms, alone_ms = max_over_ranks([total_ms, enc_ms, dec_ms, alone_ms], world)
     return {"total_ms": total_ms, "enc_ms": enc_ms, "dec_ms": dec_ms, "alone_ms": alone_ms,
             "launches": int(launches), "clocks": clocks, "clocks_alone": clocks2, "ladder": ladder,
+            "graph": graph,
             "codes": codes, "scales": scales, "out": out}
 
 
@@ -680,6 +720,8 @@ def main():
             "gpu_launches": m["launches"],
             "clocks": m["clocks"],
         }
+        if m.get("graph"):
+            line["graph_replay"] = m["graph"]
         if message:
             line["message"] = message
         if sweep is not None:

@@ -123,6 +123,37 @@ def _dev(t: torch.Tensor, dtype, name: str) -> int:
     return t.data_ptr()
 
 
+class PointerTable:
+    """Device addresses of a fixed list of tensors, checked and marshalled once.  The calls
+    that take one tensor per worker accept a table in place of the sequence, which saves the
+    per-tensor checks on every call when the same buffers serve every step.  The table keeps
+    its tensors alive; it holds addresses, so a tensor that is resized or replaced needs a new
+    table."""
+    __slots__ = ("array", "n", "dtype", "_keep")
+
+    def __init__(self, tensors: Sequence[torch.Tensor], dtype, name: str = "tensors"):
+        self._keep = list(tensors)
+        self.n = len(self._keep)
+        self.dtype = dtype
+        self.array = (ctypes.c_void_p * self.n)(*[_dev(x, dtype, name) for x in self._keep])
+
+    def __len__(self) -> int:
+        return self.n
+
+
+def pointer_table(tensors: Sequence[torch.Tensor], dtype, name: str = "tensors") -> PointerTable:
+    """Marshal a list of CUDA tensors of one dtype once, for use in many calls."""
+    return PointerTable(tensors, dtype, name)
+
+
+def _table(ts, dtype, name: str) -> PointerTable:
+    if isinstance(ts, PointerTable):
+        if ts.dtype != dtype:
+            raise ValueError("%s must be a table of %s tensors" % (name, dtype))
+        return ts
+    return PointerTable(ts, dtype, name)
+
+
 def ecq_create(d: int, bucket: int, levels: int, alpha: float, beta: float, seed: int) -> int:
     """Return an opaque context handle (see ``ecq_create`` in ecq.h)."""
     h = ctypes.c_void_p()
@@ -191,24 +222,28 @@ def ecq_encode(ctx: int, worker: int, step: int, grad: torch.Tensor, err: torch.
 def ecq_encode_batch(ctx: int, step: int, grads: Sequence[torch.Tensor],
                      errs: Sequence[torch.Tensor], codes: Sequence[torch.Tensor],
                      scales: Sequence[torch.Tensor], stream=None) -> None:
-    """Enqueue the sender-side kernel for workers 0..len(grads)-1 as one launch."""
+    """Enqueue the sender-side kernel for workers 0..len(grads)-1 as one launch.  Each of the
+    four arguments is a sequence of tensors or a ``pointer_table`` of them."""
     W = len(grads)
     if not (len(errs) == len(codes) == len(scales) == W):
         raise ValueError("grads, errs, codes and scales must have one entry per worker")
-    arr = lambda ts, dt, nm: (ctypes.c_void_p * W)(*[_dev(x, dt, nm) for x in ts])  # noqa: E731
-    rc = lib().ecq_encode_batch(ctx, W, step, arr(grads, torch.float32, "grads"),
-                                arr(errs, torch.float32, "errs"), arr(codes, torch.int32, "codes"),
-                                arr(scales, torch.float32, "scales"), _stream(stream))
+    rc = lib().ecq_encode_batch(ctx, W, step, _table(grads, torch.float32, "grads").array,
+                                _table(errs, torch.float32, "errs").array,
+                                _table(codes, torch.int32, "codes").array,
+                                _table(scales, torch.float32, "scales").array, _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_encode_batch")
 
 
 def ecq_decode_mean(ctx: int, codes: Sequence[torch.Tensor], scales: Sequence[torch.Tensor],
                     out: torch.Tensor, stream=None) -> None:
-    """Enqueue the fused receiver-side kernel over ``len(codes)`` messages."""
+    """Enqueue the fused receiver-side kernel over ``len(codes)`` messages (sequences of
+    tensors or ``pointer_table``s)."""
     W = len(codes)
-    cp = (ctypes.c_void_p * W)(*[_dev(c, torch.int32, "codes") for c in codes])
-    sp = (ctypes.c_void_p * W)(*[_dev(s, torch.float32, "scales") for s in scales])
+    if len(scales) != W:
+        raise ValueError("codes and scales must have one entry per message")
+    cp = _table(codes, torch.int32, "codes").array
+    sp = _table(scales, torch.float32, "scales").array
     rc = lib().ecq_decode_mean(ctx, W, cp, sp, _dev(out, torch.float32, "out"), _stream(stream))
     if rc != ECQ_OK:
         raise EcqError(rc, "ecq_decode_mean")
@@ -218,8 +253,10 @@ def ecq_decode_mean_update(ctx: int, codes: Sequence[torch.Tensor], scales: Sequ
                            eta: float, params: torch.Tensor, out=None, stream=None) -> None:
     """Receiver-side kernel with ``params <- params - eta * mean`` fused in."""
     W = len(codes)
-    cp = (ctypes.c_void_p * W)(*[_dev(c, torch.int32, "codes") for c in codes])
-    sp = (ctypes.c_void_p * W)(*[_dev(s, torch.float32, "scales") for s in scales])
+    if len(scales) != W:
+        raise ValueError("codes and scales must have one entry per message")
+    cp = _table(codes, torch.int32, "codes").array
+    sp = _table(scales, torch.float32, "scales").array
     rc = lib().ecq_decode_mean_update(ctx, W, cp, sp, eta, _dev(params, torch.float32, "params"),
                                       None if out is None else _dev(out, torch.float32, "out"),
                                       _stream(stream))

@@ -47,3 +47,11 @@ def test_binding_refuses_host_tensors():
     with pytest.raises(ValueError):
         binding.ecq_encode(1, 0, 0, torch.zeros(4), torch.zeros(4),
                            torch.zeros(1, dtype=torch.int32), torch.zeros(1))
+
+
+def test_pointer_table_refuses_host_tensors_and_wrong_types():
+    import torch
+    with pytest.raises(ValueError):
+        binding.pointer_table([torch.zeros(4)], torch.float32, "grads")
+    with pytest.raises(ValueError):
+        binding.ecq_decode_mean(1, [torch.zeros(1, dtype=torch.int32)], [], torch.zeros(4))

@@ -55,6 +55,8 @@ def test_own_arm_line():
         assert ca["kind"] == "oracle" and ca["cores"] == min(8, os.cpu_count()) and ca["value"] > 0
     assert "sweep" not in j                                 # only the default workload carries it
     assert dec["length_ladder"] is None                     # shorter than two rounds of long-vector tiles
+    gr = j["graph_replay"]                                  # an L2-resident workload: also as one CUDA graph
+    assert gr["steps_per_graph"] == 3 and 0 < gr["ms_per_step"] <= j["ms_per_step"] * 1.5 and gr["GB/s"] > 0
 
 
 def test_receiver_length_ladder_on_a_mid_size_workload():
@@ -62,6 +64,7 @@ def test_receiver_length_ladder_on_a_mid_size_workload():
              "--no-message")
     lad = j["decode"]["length_ladder"]
     assert lad["rounds"] == [1, 2, 3, 4] and lad["entries_per_round"] % 30720 == 0
+    assert "graph_replay" not in j                          # larger than L2: the plain loop is the measure
     for name in ("ring", "warp"):
         k = lad[name]
         assert len(k["us"]) == 4 and all(u > 0 for u in k["us"])

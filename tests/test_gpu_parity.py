@@ -503,3 +503,37 @@ def test_code_width_matched_levels_on_resnet50():
     base = wl.WORKLOADS["resnet50"]
     for s in (3, 7, 127):
         _sampled_config(wl.with_codec(base, base.bucket, s), steps=1, W=2)
+
+
+def test_pointer_tables_give_the_same_launches_as_tensor_lists():
+    # the binding marshals a fixed list of tensors once; the calls are the same
+    d, bucket, s_, W = 300_000 + 40, 512, 4, 4
+    gpu = GpuCodec(d, bucket, s_, 1.0, 0.9, SEED, W)
+    gen = torch.Generator(device="cuda"); gen.manual_seed(3)
+    grads = [0.01 * torch.randn(d, generator=gen, device="cuda") for _ in range(W)]
+    gpu.encode_batch(0, grads)
+    gpu.decode()
+    want_codes = [c[1].clone() for c in gpu.codes]
+    want_err = [e[1].clone() for e in gpu.err]
+    want_out = gpu.out[1].clone()
+    for e in gpu.err:
+        e[1].zero_()
+    tg = ecq.pointer_table(grads, torch.float32, "grads")
+    te = ecq.pointer_table([e[1] for e in gpu.err], torch.float32, "errs")
+    tc = ecq.pointer_table([c[1] for c in gpu.codes], torch.int32, "codes")
+    ts = ecq.pointer_table([x[1] for x in gpu.scales], torch.float32, "scales")
+    assert len(tc) == W
+    for c in gpu.codes:
+        c[1].zero_()
+    gpu.out[1].zero_()
+    ecq.ecq_encode_batch(gpu.ctx, 0, tg, te, tc, ts)
+    ecq.ecq_decode_mean(gpu.ctx, tc, ts, gpu.out[1])
+    assert gpu.status() == ecq.ECQ_OK
+    for w in range(W):
+        assert torch.equal(gpu.codes[w][1], want_codes[w])
+        assert torch.equal(gpu.err[w][1].view(torch.int32), want_err[w].view(torch.int32))
+    assert torch.equal(gpu.out[1].view(torch.int32), want_out.view(torch.int32))
+    with pytest.raises(ValueError):
+        ecq.ecq_decode_mean(gpu.ctx, ts, ts, gpu.out[1])           # a table of the wrong type
+    gpu.check_guards()
+    gpu.close()
