@@ -244,7 +244,14 @@ __device__ __forceinline__ void decode_ring_consumer(
     const uint32_t gsz = P.bucket >= 1024u ? 32u : (P.bucket >> 5);
     const uint32_t gl = lane & (gsz - 1);
     const uint32_t bucket_shift = 31 - __clz(P.bucket);           // bucket is a power of two
-    const uint32_t n_slots = (W + gsz - 1) / gsz;                   // <= kDecAreg
+    // Level steps enter the tables as a_w 2^-22 (against the 2^p of the fields) and, when the
+    // whole mean is taken here over a power-of-two number of messages, divided by it as well:
+    // powers of two, so the chain's roundings are those of Eq. 4 and the stored mean needs one
+    // multiply.  With s a power of two the division scale / s is a multiplication too.
+    const bool pre_w = !CARRY && w_pow2;
+    const bool s_pow2 = (P.s & (P.s - 1u)) == 0u;
+    const float k_pre = pre_w ? __fmul_rn(0x1p-22f, w_recip) : 0x1p-22f;
+    const float a_mul = s_pow2 ? __fdiv_rn(k_pre, P.sf) : k_pre;
     const uint32_t grp = L::kFixedLayout ? (lane & ~(gsz - 1)) * kDecAreg : ((uint32_t)lane / gsz) * lay.wstride;   // my group's first entry
     const uint32_t raw_u32 = smem_u32(raw);
 
@@ -266,12 +273,9 @@ __device__ __forceinline__ void decode_ring_consumer(
             const uint32_t sub = tile * kRingSubs + warp + row * kRingWarps;
             if (sub < n_subs) {
                 const uint64_t b = ((uint64_t)sub * kDecTileElems + (uint32_t)lane * 32) >> bucket_shift;
-#pragma unroll
-                for (int k = 0; k < kDecAreg; ++k) {
-                    const uint32_t w = k * gsz + gl;
-                    if (k < (int)n_slots && w < W)
-                        cp_async4(raw_u32 + ((grp + w) * 2 + row) * 4, tab.scales[w] + b);
-                }
+#pragma unroll 1
+                for (uint32_t w = gl; w < W; w += gsz)
+                    cp_async4(raw_u32 + ((grp + w) * 2 + row) * 4, tab.scales[w] + b);
             }
         }
         cp_async_commit();
@@ -335,14 +339,12 @@ __device__ __forceinline__ void decode_ring_consumer(
         // bits, far under the absolute tolerance) against the 2^(iR) of the fields
         cp_async_wait<0>();
         __syncwarp();
-#pragma unroll
-        for (int k = 0; k < kDecAreg; ++k) {
-            const uint32_t w = k * gsz + gl;
-            if (k < (int)n_slots && w < W) {
-                const float2 sc = *reinterpret_cast<const float2*>(raw + (grp + w) * 2);
-                a_tab[grp + w] = make_float2(__fmul_rn(__fdiv_rn(sc.x, P.sf), 0x1p-22f),
-                                             __fmul_rn(__fdiv_rn(sc.y, P.sf), 0x1p-22f));
-            }
+#pragma unroll 1
+        for (uint32_t w = gl; w < W; w += gsz) {
+            const float2 sc = *reinterpret_cast<const float2*>(raw + (grp + w) * 2);
+            a_tab[grp + w] = s_pow2 ? make_float2(__fmul_rn(sc.x, a_mul), __fmul_rn(sc.y, a_mul))
+                                    : make_float2(__fmul_rn(__fdiv_rn(sc.x, P.sf), a_mul),
+                                                  __fmul_rn(__fdiv_rn(sc.y, P.sf), a_mul));
         }
         __syncwarp();
         if (ti + 1 < my_tiles) fetch_scales(tile + gridDim.x);
@@ -401,7 +403,7 @@ __device__ __forceinline__ void decode_ring_consumer(
                     float lo, hi;
                     unpack2(acc2[j], lo, hi);
                     const float x = __fmul_rn(row ? hi : lo, __uint_as_float((uint32_t)(127 + 22 - L::field_shift(j)) << 23));
-                    v[k] = !last ? x : w_pow2 ? __fmul_rn(x, w_recip) : __fdiv_rn(x, w_total);
+                    v[k] = (!last || pre_w) ? x : w_pow2 ? __fmul_rn(x, w_recip) : __fdiv_rn(x, w_total);
                 }
                 if (last) emit8(dst, o + 8 * c, v);
                 else stg256(dst.out + o + 8 * c, v);
