@@ -213,6 +213,14 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
     const uint32_t bucket_shift = 31 - __clz(P.bucket);           // bucket is a power of two
     const uint32_t n_slots = (W + gsz - 1) / gsz;                   // <= kDecAreg
     float2* const a_mine = a_tab + (lane / gsz) * (kDecAreg * gsz);
+    // Level steps enter the table as a_w 2^-22 (against the 2^(iR) of the fields) and, when the
+    // whole mean is taken here over a power-of-two number of messages, divided by it as well:
+    // powers of two, so the chain's roundings are those of Eq. 4 and the stored mean needs one
+    // multiply.  With s a power of two the division scale / s is a multiplication too.
+    const bool pre_w = !CARRY && w_pow2;
+    const bool s_pow2 = (P.s & (P.s - 1u)) == 0u;
+    const float k_pre = pre_w ? __fmul_rn(0x1p-22f, w_recip) : 0x1p-22f;
+    const float a_mul = s_pow2 ? __fdiv_rn(k_pre, P.sf) : k_pre;
 
     // 2^23 + s * 2^(iR): subtracting it from (field | 0x4B000000) leaves (c - s) * 2^(iR)
     uint64_t T2[FIT / 2];
@@ -271,7 +279,7 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
 #pragma unroll
         for (int k = 0; k < kDecAreg; ++k)
             if (k < (int)n_slots) {
-                const float a = __fmul_rn(__fdiv_rn(nxt[k], P.sf), 0x1p-22f);
+                const float a = s_pow2 ? __fmul_rn(nxt[k], a_mul) : __fmul_rn(__fdiv_rn(nxt[k], P.sf), a_mul);
                 a_mine[k * gsz + gl] = make_float2(a, a);
             }
         __syncwarp();
@@ -356,7 +364,7 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         float acc[32];
 #pragma unroll
         for (int j = 0; j < 16; ++j) unpack2(acc2[j], acc[2 * j], acc[2 * j + 1]);
-        if (!last) {
+        if (!last || pre_w) {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
                 acc[j] = __fmul_rn(acc[j], __uint_as_float((uint32_t)(127 + 22 - (j % FIT) * R) << 23));
