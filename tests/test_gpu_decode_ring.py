@@ -87,6 +87,17 @@ def test_scales_near_one_stay_within_tolerance():
                 decode_plan=(ecq.ECQ_DECODE_RING, 2))
 
 
+@pytest.mark.parametrize("scale", [1e30, 1e-33])
+@pytest.mark.parametrize("plan", [(ecq.ECQ_DECODE_RING, 2), (ecq.ECQ_DECODE_WARP, 0)])
+def test_very_large_and_very_small_gradients(scale, plan):
+    # the kernels carry the level steps times 2^-22 / W: sums near the top of the fp32 range must
+    # not overflow on the way, and level steps that fall below the normal range may lose bits
+    # only far under the absolute tolerance
+    d, bucket, s, W = TILE * 2 + 1024 * 7 + 3, 512, 4, 8
+    full_parity(d, bucket, s, 1.0, 0.9, SEED, W=W, steps=1, grad_fn=randn_fn(d, scale=scale, base=9),
+                decode_plan=plan)
+
+
 def test_every_kernel_gives_the_same_bits_on_a_long_vector():
     # any size: the kernels sum in the same order, so their outputs are bit-identical
     w = wl.WORKLOADS["resnet50"]
