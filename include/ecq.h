@@ -191,7 +191,10 @@ int ecq_encode_batch(ecq_ctx* ctx, uint32_t W, uint32_t step, const float* const
  * messages are summed in one launch; beyond that there is one launch per
  * ECQ_MAX_WORKERS messages, each continuing the sum of the previous one (kept in
  * `out` meanwhile) in the same ascending order of w, so the result is the same
- * chain of fp32 operations as a single pass.
+ * chain of fp32 operations as a single pass.  The long-vector kernels carry the
+ * level steps times a power of two (2^-22, and 1/W when W is a power of two):
+ * exact, except that level steps below 2^-94 may lose low-order bits, an error
+ * far below any gradient that matters.
  */
 int ecq_decode_mean(ecq_ctx* ctx, uint32_t W, const uint32_t* const* codes,
                     const float* const* scales, float* out, void* cuda_stream);
