@@ -6,6 +6,14 @@
 
 namespace ecq {
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start while its predecessor in the stream still runs; it must not touch global memory
+// before griddep_wait() (which returns once the predecessor has completed and its writes are
+// visible).  griddep_launch() lets the successor's CTAs be scheduled as this grid's leave.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
 constexpr uint32_t kStatusNonFinite = 1u;   // device status word bits
 constexpr uint32_t kStatusTimeout = 2u;
 

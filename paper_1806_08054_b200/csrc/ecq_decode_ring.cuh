@@ -456,7 +456,9 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         *reinterpret_cast<volatile uint32_t*>(dsm + 264) = 0;
         fence_mbar_init();
     }
+    griddep_launch();
     __syncthreads();
+    griddep_wait();
 
     if (warp == kRingWarps) {
         // ---- producer: fill n = my n / n_groups-th tile, workers G (n % n_groups) and up, in

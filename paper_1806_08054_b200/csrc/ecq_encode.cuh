@@ -238,6 +238,8 @@ encode_tiled_kernel(const __grid_constant__ EncodeBatch bt, const CodecParams P,
         tma_load_2d(base + L::kLoadOff, &bt.tm_g[e], 0, (int)(tile * kTileRows), bar_full);
         tma_load_2d(base + L::kLoadOff + kTileBytes, &bt.tm_h[e], 0, (int)(tile * kTileRows), bar_full);
     };
+    griddep_launch();
+    griddep_wait();
     if (tid == 0) {
         mbar_init(bar_full, 1);
         *s_abort = 0;
