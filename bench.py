@@ -456,9 +456,11 @@ def measure(ecq, ctx, w, grad_list, errs, steps, warmup, rank, local, world, lad
     # the receiver kernel by itself: launches back to back (its inputs stay as the last step
     # left them) after a short idle, so that it is not timed at the clock a long, power-capped
     # encode left behind; the clock sampled during these launches is reported beside the time
-    n_alone = max(3, min(20, int(4.0 / max(dec_ms / steps, 1e-3))))
+    # (about 10 ms of launches, half as many before them: a handful of 50 us launches right
+    # after the idle would be timed while the clock is still coming up)
+    n_alone = max(3, min(200, int(10.0 / max(dec_ms / steps, 1e-3))))
     time.sleep(0.3)
-    for _ in range(2):
+    for _ in range(max(2, n_alone // 2)):
         ecq.ecq_decode_mean(ctx, t_c, t_s, out)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -321,8 +321,8 @@ bool launch_decode_ring(ecq_ctx* c, uint32_t W, const MessageTable& tab, DecodeO
     if (lay.stages < 3) return false;
     const uint32_t full = (uint32_t)(c->sm_count * occ[dev]);
     uint32_t grid = full;
-    if (c->decode_kernel == ECQ_DECODE_AUTO &&
-        (n_tiles < (uint64_t)kRingMinTilesPerCta * grid || R > kRingMaxAutoBits))
+    const uint64_t min_tiles_per_cta = (uint64_t)ring_min_tiles_per_cta(R, W);
+    if (c->decode_kernel == ECQ_DECODE_AUTO && (n_tiles < min_tiles_per_cta * grid || R > kRingMaxAutoBits))
         return false;
     if (c->decode_max_ctas && grid > c->decode_max_ctas) grid = c->decode_max_ctas;
     if (grid > n_tiles) grid = (uint32_t)n_tiles;

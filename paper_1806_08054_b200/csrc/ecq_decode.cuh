@@ -135,6 +135,50 @@ decode_mean_generic_kernel(const CodecParams P, const uint32_t W,
 }
 
 
+// Ragged end of a vector behind its last whole tile of 1024 outputs: one thread per output,
+// the chain of Eq. 4 as in decode_mean_generic_kernel.  The loads of eight messages are issued
+// before the first of them is used (one message at a time, each turn of the loop waits for a
+// trip to DRAM: 32 messages kept the last CTA 10 us beyond the others), and the outputs go to
+// the CTAs from the end of the grid, which are the ones with the fewest tiles.
+template <int R>
+__device__ __forceinline__ void decode_ragged_end(const CodecParams& P, const uint32_t W,
+                                                  const MessageTable& tab, const DecodeOut& dst,
+                                                  const uint64_t tail0, const uint64_t n_words,
+                                                  const bool first, const bool last, const float w_recip,
+                                                  const int w_pow2, const float w_total) {
+    constexpr uint32_t mask = (1u << R) - 1u;
+    const float magic = 8388608.f + P.sf;
+    const uint32_t rev = gridDim.x - 1u - blockIdx.x;
+    for (uint64_t i = tail0 + (uint64_t)rev * blockDim.x + threadIdx.x; i < P.d;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t b = i / P.bucket, bit = i * R, wi = bit >> 5;
+        const uint32_t sh = (uint32_t)(bit & 31);
+        const bool two = sh + R > 32 && wi + 1 < n_words;
+        float acc1 = first ? 0.f : dst.out[i];
+        for (uint32_t w0 = 0; w0 < W; w0 += 8) {
+            float sc[8];
+            uint32_t lo[8], hi[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const bool in = w0 + k < W;
+                sc[k] = in ? __ldg(tab.scales[w0 + k] + b) : 0.f;
+                lo[k] = in ? __ldg(tab.codes[w0 + k] + wi) : 0u;
+                hi[k] = (in && two) ? __ldg(tab.codes[w0 + k] + wi + 1) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (w0 + k < W) {
+                    const float a = __fdiv_rn(sc[k], P.sf);
+                    const uint32_t c = __funnelshift_r(lo[k], hi[k], sh) & mask;
+                    acc1 = __fmaf_rn(__fsub_rn(__uint_as_float(0x4B000000u | c), magic), a, acc1);
+                }
+            }
+        }
+        if (!last) dst.out[i] = acc1;
+        else emit1(dst, i, w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, w_total));
+    }
+}
+
 // ===========================================================================
 // Tiled path.  Every warp works on its own: a tile is 1024 outputs, one run of
 // 32 consecutive entries ("row") per lane, whose codes are R whole words.
@@ -403,24 +447,8 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
     }
     cp_async_wait<0>();
 
-    // ragged end (fewer than 1024 outputs): one thread per output
-    const uint64_t tail0 = (uint64_t)n_tiles * kDecTileElems;
-    const float magic = 8388608.f + P.sf;
-    for (uint64_t i = tail0 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < P.d;
-         i += (uint64_t)gridDim.x * blockDim.x) {
-        const uint64_t b = i / P.bucket, bit = i * R, wi = bit >> 5;
-        const uint32_t sh = (uint32_t)(bit & 31);
-        float acc1 = first ? 0.f : dst.out[i];
-        for (uint32_t w = 0; w < W; ++w) {
-            const float a = __fdiv_rn(__ldg(tab.scales[w] + b), P.sf);
-            const uint32_t lo = __ldg(tab.codes[w] + wi);
-            const uint32_t hi1 = (sh + R > 32 && wi + 1 < n_words) ? __ldg(tab.codes[w] + wi + 1) : 0u;
-            const uint32_t c = __funnelshift_r(lo, hi1, sh) & mask;
-            acc1 = __fmaf_rn(__fsub_rn(__uint_as_float(0x4B000000u | c), magic), a, acc1);
-        }
-        if (!last) dst.out[i] = acc1;
-        else emit1(dst, i, w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, w_total));
-    }
+    decode_ragged_end<R>(P, W, tab, dst, (uint64_t)n_tiles * kDecTileElems, n_words, first, last, w_recip,
+                         w_pow2, w_total);
 }
 
 }  // namespace ecq

@@ -40,10 +40,19 @@ constexpr int kRingThreads = (kRingWarps + 1) * 32;
 constexpr int kRingSubs = 2 * kRingWarps;                       // sub-tiles per CTA tile
 constexpr int kRingTileElems = kRingSubs * kDecTileElems;       // 30720 outputs
 // What the automatic choice asks for: shorter vectors leave the CTAs with too uneven a share
-// of these large tiles (measured: 7 % slower than the warp-tiled kernel at 5.6 tiles per CTA,
-// 7 % faster at 13, 10 % faster at 78), and at r = 9 the receiver is bound by HBM, not by
-// instruction issue, where the warp-tiled kernel's deeper private rings do better.
+// of these large tiles (a CTA's time goes by whole tiles), and at r = 9 the receiver is bound
+// by HBM, not by instruction issue, where the warp-tiled kernel's deeper private rings do
+// better.  With few messages of wide codes the vector has to be long:
 constexpr int kRingMinTilesPerCta = 12;
+// The more messages and the narrower the codes, the smaller the per-tile work (level steps,
+// stores) is beside the per-code work, and the sooner this kernel is ahead.  Measured on
+// vectors of 1.2 / 2.1 / 3.3 / 5.6 tiles per CTA, time of this kernel over the warp-tiled one:
+// 32 messages of 4 bits 1.00 / 0.96 / 0.81 / 0.77, 16 of 4 bits 1.10 / 1.01 / 0.89 / 0.83,
+// 8 of 4 bits 1.05 / 1.19 / 1.05 / 0.98, 32 of 5 bits 1.17 / 1.18 / 0.99 / 0.93, 8 of 5 bits
+// 1.19 / 1.31 / 1.10 / 1.04, 4 messages always above 1.
+__host__ __device__ constexpr int ring_min_tiles_per_cta(int r, uint32_t W) {
+    return (r <= 4 && W >= 16) ? 3 : ((r <= 4 && W >= 8) || W >= 16) ? 5 : kRingMinTilesPerCta;
+}
 constexpr int kRingMaxAutoBits = 8;
 
 template <int R> struct DecodeRing {
@@ -432,7 +441,6 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
     const bool first = CARRY ? sl.first != 0 : true, last = CARRY ? sl.last != 0 : true;
     const float w_total = CARRY ? sl.w_total : (float)W;
     const uint32_t S = L::kFixedLayout ? (uint32_t)L::kFixedStages : lay.stages;
-    constexpr uint32_t mask = (1u << R) - 1u;
     extern __shared__ __align__(128) uint8_t dsm[];
     const uint32_t sm0 = smem_u32(dsm);
     const uint32_t bar_full = sm0, bar_empty = sm0 + 128;
@@ -505,24 +513,8 @@ decode_ring_kernel(const CodecParams P, const uint32_t W, const __grid_constant_
         return;
     }
 
-    // ragged end (fewer than 1024 outputs): one thread per output
-    const uint64_t tail0 = (uint64_t)n_subs * kDecTileElems;
-    const float magic = 8388608.f + P.sf;
-    for (uint64_t i = tail0 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < P.d;
-         i += (uint64_t)gridDim.x * blockDim.x) {
-        const uint64_t b = i / P.bucket, bit = i * R, wi = bit >> 5;
-        const uint32_t sh = (uint32_t)(bit & 31);
-        float acc1 = first ? 0.f : dst.out[i];
-        for (uint32_t w = 0; w < W; ++w) {
-            const float a = __fdiv_rn(__ldg(tab.scales[w] + b), P.sf);
-            const uint32_t lo = __ldg(tab.codes[w] + wi);
-            const uint32_t hi1 = (sh + R > 32 && wi + 1 < n_words) ? __ldg(tab.codes[w] + wi + 1) : 0u;
-            const uint32_t c = __funnelshift_r(lo, hi1, sh) & mask;
-            acc1 = __fmaf_rn(__fsub_rn(__uint_as_float(0x4B000000u | c), magic), a, acc1);
-        }
-        if (!last) dst.out[i] = acc1;
-        else emit1(dst, i, w_pow2 ? __fmul_rn(acc1, w_recip) : __fdiv_rn(acc1, w_total));
-    }
+    decode_ragged_end<R>(P, W, tab, dst, (uint64_t)n_subs * kDecTileElems, n_words, first, last, w_recip,
+                         w_pow2, w_total);
 }
 
 }  // namespace ecq
