@@ -45,9 +45,9 @@ NOMINAL_HBM_GBS = 8000.0
 # proportion to the entries of a launch, so a full launch's traffic is this figure times its
 # entries.  An entry is dropped (traffic: null) when the kernel changes until it is re-taken.
 NCU_DRAM_BYTES_PER_ENTRY = {      # (bucket, levels): bytes per entry, read + write
-    (512, 4): 10185023744 / 817825024, (128, 1): 9999779584 / 817825024,
-    (4096, 8): 10280564480 / 817825024, (4096, 128): 10688161792 / 817825024,
-    (512, 8): 10285686784 / 817825024, (2048, 1): 9976081408 / 817825024,
+    (512, 4): 10185571840 / 817825024, (128, 1): 9999337984 / 817825024,
+    (4096, 8): 10281645056 / 817825024, (4096, 128): 10688185856 / 817825024,
+    (512, 8): 10285809408 / 817825024, (2048, 1): 9976462848 / 817825024,
 }
 
 

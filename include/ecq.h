@@ -12,7 +12,10 @@
  *     by the caller; the library never frees or reallocates them.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL
  *     is the default stream) and the call returns without synchronising,
- *     unless stated otherwise.
+ *     unless stated otherwise.  Stream order is kept: a kernel of this library
+ *     may be scheduled while the work ahead of it in the stream is finishing
+ *     (programmatic dependent launch), but touches no global memory before
+ *     that work has completed, so buffers may be reused from call to call.
  *   - `grad`, `err`, `out`, `codes` must be 16-byte aligned; `scales` 4-byte.
  *   - A context is immutable after creation (except the ecq_set_* calls) and may
  *     be used from several host threads on different streams.
@@ -106,7 +109,9 @@ int ecq_set_norm(ecq_ctx* ctx, int norm);
  *   kernel    ECQ_DECODE_AUTO (default): by shape and length;
  *             ECQ_DECODE_WARP: tiles of 1024 outputs, every warp copies its own code words;
  *             ECQ_DECODE_RING: tiles of 30720 outputs, one bulk copy per (tile, worker)
- *             shared by the CTA (what AUTO takes for long vectors with r <= 8).
+ *             shared by the CTA (what AUTO takes for r <= 8 once a CTA has enough tiles:
+ *             3 with 16 messages or more of up to 4 bits, 5 with 8 or more of up to 4 bits
+ *             or 16 or more of up to 8 bits, 12 otherwise).
  *             A shape that a kernel does not cover (bucket not a power of two, r > 9, more
  *             than bucket/4 workers for buckets under 1024; for RING also `out` or
  *             `params` not 32-byte aligned) falls through to the next one.
