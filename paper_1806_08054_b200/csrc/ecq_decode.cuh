@@ -307,8 +307,15 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         cp_async_commit();
     };
     // ---- scales of my bucket for one tile: worker k*gsz + gl in slot k ----
+    // (With no more messages than lanes in a group -- the usual case -- a lane has one slot:
+    // the unrolled loop over all eight would issue its predicated-off instructions all the
+    // same, which shows once the per-tile work is spread over few messages.)
     auto load_scales = [&](uint32_t tile, float (&dst)[kDecAreg]) {
         const uint64_t b = ((uint64_t)tile * kDecTileElems + (uint32_t)lane * 32) >> bucket_shift;
+        if (n_slots == 1) {
+            dst[0] = (gl < W) ? __ldg(tab.scales[gl] + b) : 0.f;
+            return;
+        }
 #pragma unroll
         for (int k = 0; k < kDecAreg; ++k) {
             if (k < (int)n_slots) {
@@ -328,12 +335,17 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
         const uint32_t tile = gw + ti * n_warps;
         // a_w = scale_w / s, pre-scaled by 2^-22 (exact; only scales below 2^-104 lose
         // bits, far under the absolute tolerance) against the 2^(iR) of the fields
+        if (n_slots == 1) {
+            const float a = s_pow2 ? __fmul_rn(nxt[0], a_mul) : __fmul_rn(__fdiv_rn(nxt[0], P.sf), a_mul);
+            a_mine[gl] = make_float2(a, a);
+        } else {
 #pragma unroll
-        for (int k = 0; k < kDecAreg; ++k)
-            if (k < (int)n_slots) {
-                const float a = s_pow2 ? __fmul_rn(nxt[k], a_mul) : __fmul_rn(__fdiv_rn(nxt[k], P.sf), a_mul);
-                a_mine[k * gsz + gl] = make_float2(a, a);
-            }
+            for (int k = 0; k < kDecAreg; ++k)
+                if (k < (int)n_slots) {
+                    const float a = s_pow2 ? __fmul_rn(nxt[k], a_mul) : __fmul_rn(__fdiv_rn(nxt[k], P.sf), a_mul);
+                    a_mine[k * gsz + gl] = make_float2(a, a);
+                }
+        }
         __syncwarp();
         if (ti + 1 < my_tiles) load_scales(tile + n_warps, nxt);
 
@@ -436,12 +448,21 @@ decode_tiled_kernel(const CodecParams P, const uint32_t W, const __grid_constant
                 make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
         __syncwarp();
         const uint64_t o = (uint64_t)tile * kDecTileElems;
+        if (last && dst.params) {
+            // with the fused model update (one branch per tile, not a predicate per store)
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
-            const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
-            if (last) emit4(dst, o + idx * 4, v);
-            else *reinterpret_cast<float4*>(dst.out + o + idx * 4) = v;
+            for (int k = 0; k < 8; ++k) {
+                const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
+                const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
+                emit4(dst, o + idx * 4, v);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int idx = k * 32 + lane, row = idx >> 3, ch = idx & 7;
+                const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
+                *reinterpret_cast<float4*>(dst.out + o + idx * 4) = v;
+            }
         }
         __syncwarp();
     }
