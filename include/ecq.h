@@ -110,8 +110,8 @@ int ecq_set_norm(ecq_ctx* ctx, int norm);
  *             ECQ_DECODE_WARP: tiles of 1024 outputs, every warp copies its own code words;
  *             ECQ_DECODE_RING: tiles of 30720 outputs, one bulk copy per (tile, worker)
  *             shared by the CTA (what AUTO takes for r <= 8 once a CTA has enough tiles:
- *             3 with 16 messages or more of up to 4 bits, 5 with 8 or more of up to 4 bits
- *             or 16 or more of up to 8 bits, 12 otherwise).
+ *             3 with 12 messages or more of up to 4 bits, 5 with 8 or more of 2 bits or
+ *             12 or more of up to 8 bits, 12 otherwise).
  *             A shape that a kernel does not cover (bucket not a power of two, r > 9, more
  *             than bucket/4 workers for buckets under 1024; for RING also `out` or
  *             `params` not 32-byte aligned) falls through to the next one.

@@ -46,12 +46,13 @@ constexpr int kRingTileElems = kRingSubs * kDecTileElems;       // 30720 outputs
 constexpr int kRingMinTilesPerCta = 12;
 // The more messages and the narrower the codes, the smaller the per-tile work (level steps,
 // stores) is beside the per-code work, and the sooner this kernel is ahead.  Measured on
-// vectors of 1.2 / 2.1 / 3.3 / 5.6 tiles per CTA, time of this kernel over the warp-tiled one:
-// 32 messages of 4 bits 1.00 / 0.96 / 0.81 / 0.77, 16 of 4 bits 1.10 / 1.01 / 0.89 / 0.83,
-// 8 of 4 bits 1.05 / 1.19 / 1.05 / 0.98, 32 of 5 bits 1.17 / 1.18 / 0.99 / 0.93, 8 of 5 bits
-// 1.19 / 1.31 / 1.10 / 1.04, 4 messages always above 1.
+// vectors of 3.3 / 5.6 / 8.8 tiles per CTA, time of this kernel over the warp-tiled one:
+// 16 messages of 2 bits 0.84 / 0.77 / 0.74, of 4 bits 0.94 / 0.88 / 0.86, of 5 bits 1.04 / 0.97 /
+// 0.97; 12 messages the same within 0.03; 8 messages of 2 bits 1.00 / 0.93 / 0.89, of 4 bits
+// 1.14 / 1.07 / 1.00, of 5 bits 1.19 / 1.10 / 1.02; 32 messages of 4 bits 0.81 / 0.77 and 0.96
+// at 2.1 tiles; 4 messages always above 1.
 __host__ __device__ constexpr int ring_min_tiles_per_cta(int r, uint32_t W) {
-    return (r <= 4 && W >= 16) ? 3 : ((r <= 4 && W >= 8) || W >= 16) ? 5 : kRingMinTilesPerCta;
+    return (r <= 4 && W >= 12) ? 3 : ((r <= 2 && W >= 8) || W >= 12) ? 5 : kRingMinTilesPerCta;
 }
 constexpr int kRingMaxAutoBits = 8;
 
