@@ -115,6 +115,27 @@ def test_every_kernel_gives_the_same_bits_on_a_long_vector():
     assert torch.equal(outs[0].view(torch.int32), outs[2].view(torch.int32))
 
 
+@pytest.mark.parametrize("bucket,s,W", [(512, 4, 16), (512, 1, 8), (4096, 8, 12)])
+def test_automatic_choice_gives_the_same_bits_on_vectors_of_a_few_tiles_per_cta(bucket, s, W):
+    # 5.6 ring tiles per CTA: with this many messages of these widths the automatic choice takes
+    # the ring kernel, with fewer or wider ones the warp-tiled kernel; the bits are the same,
+    # ragged end of 40 outputs included
+    d = wl.WORKLOADS["resnet50"].d
+    fn = randn_fn(d, base=3 * W + s)
+    grads = [fn(w, 0) for w in range(W)]
+    outs = []
+    for plan in ((ecq.ECQ_DECODE_WARP, 0), (ecq.ECQ_DECODE_RING, 0), (ecq.ECQ_DECODE_AUTO, 0)):
+        gpu = GpuCodec(d, bucket, s, 1.0, 0.9, SEED, W, decode_plan=plan)
+        gpu.encode_batch(0, grads)
+        gpu.decode()
+        assert gpu.status() == ecq.ECQ_OK
+        gpu.check_guards()
+        outs.append(gpu.out[1].clone())
+        gpu.close()
+    assert torch.equal(outs[0].view(torch.int32), outs[1].view(torch.int32))
+    assert torch.equal(outs[0].view(torch.int32), outs[2].view(torch.int32))
+
+
 def test_plan_argument_errors():
     ctx = ecq.ecq_create(4096, 512, 4, 1.0, 0.9, SEED)
     with pytest.raises(ecq.EcqError):
